@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the QuEST quantized-linear forward hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--had-block G]
+
+One "step" is one pass of the whole path (Algorithm 1: quantize X, quantize W, low-bit GEMM with
+the dequantising epilogue) through the C ABI call ``quest_linear_fwd`` on the 1.6B-scale layer:
+X[4096 x 2048] bf16, W[2048 x 2048] bf16, b = 4, Hadamard block 128 (seeded synthetic data).
+The step rotates over a ring of buffer sets larger than L2, so every step streams from HBM.
+
+Prints ONE JSON line (rank 0).  ``value`` is tokens/s with inputs resident in HBM; ``e2e`` is the
+same metric with the host->device copy of X and W and the device->host copy of y inside the
+timed region.  ``--impl reference`` times the CPU oracle instead (rank 0 only).
+
+With N > 1 (torchrun) every rank runs an independent replica of the same layer on its own GPU:
+the path has no exchange step, so there is no collective in the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "QuEST W4A4 linear fwd tokens/s"
+UNIT = "tokens/s"
+TOKENS, HIDDEN, OUT, BITS = 4096, 2048, 2048, 4
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 : dense bf16 tensor throughput (4.5 : 2.25 PFLOP/s)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, taken from the
+# committed ncu summary (profiles/); None until a capture exists.
+GEMM_DRAM_TRAFFIC_BYTES = None
+QUANT_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def workload_config(had_block: int) -> dict:
+    return {"workload": "config 2: W4A4 linear fwd, X[4096x2048] bf16 x W[2048x2048] bf16, b=4",
+            "tokens": TOKENS, "K": HIDDEN, "N": OUT, "bits": BITS, "had_block": had_block,
+            "trust_factor": 1.0, "weights": "quantized every step (Algorithm 1 as written)"}
+
+
+def quantizer_bytes(rows: int, cols: int, bits: int, in_bytes: int = 2) -> float:
+    """Algorithmic bytes of one quantizer launch: input + packed codes + mask bitmap + scales."""
+    container = 1 if bits == 1 else 2 if bits == 2 else 4 if bits <= 4 else 8
+    return rows * cols * (in_bytes + container / 8.0 + 1.0 / 8.0) + 4.0 * rows
+
+
+# ------------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._idx, self._period = device_index, period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self._period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self) -> dict:
+        s = sorted(self.samples)
+        med = s[len(s) // 2] if s else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ------------------------------------------------------------------------------------ ranks
+
+def init_ranks(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def max_over_ranks(value: float, world: int, backend_device=None) -> float:
+    """Max of a scalar over all ranks (identity at world size 1)."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=backend_device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank_step: int, steps: int, world: int, max_elapsed_s: float) -> float:
+    """Whole-job throughput of independent replicas: all ranks' tokens over the slowest rank's time."""
+    return tokens_per_rank_step * steps * world / max_elapsed_s
+
+
+# ------------------------------------------------------------------------------------ oracle legs
+
+_CFG2 = None
+
+
+def time_oracle(sample_tokens: int, had_block: int, repeats: int = 1):
+    """The CPU oracle, as it stands, on a bounded sample of the workload: `sample_tokens` rows of X
+    against the full W.  Returns (seconds per sample, threads used)."""
+    import numpy as np
+    from oracle import quest_oracle as qo
+    from paper_2502_05003_b200 import synth
+    global _CFG2
+    if _CFG2 is None:
+        _CFG2 = synth.config2()
+    cfg = _CFG2
+    x = np.ascontiguousarray(cfg["x"][:sample_tokens])
+    w = cfg["w"]
+    qo.lib()
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        qo.linear_fwd(x, w, BITS, had_block, 1.0)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    threads = int(os.environ.get("OMP_NUM_THREADS", "0")) or (os.cpu_count() or 1)
+    return best, threads
+
+
+def run_reference(args, rank: int):
+    if rank != 0:
+        return
+    # size the per-step sample so that the whole run stays near a minute: calibrate on 64 rows
+    sample = args.ref_tokens
+    if sample <= 0:
+        t64, _ = time_oracle(64, args.had_block)
+        t128, _ = time_oracle(128, args.had_block)
+        per_token = max((t128 - t64) / 64.0, 1e-6)
+        fixed = max(t64 - 64 * per_token, 0.0)
+        budget = 75.0 / max(args.steps + args.warmup, 1) - fixed
+        sample = int(min(TOKENS, max(8, budget / per_token)))
+        sample -= sample % 8
+    times = []
+    threads = 1
+    for i in range(args.warmup + args.steps):
+        dt, threads = time_oracle(sample, args.had_block)
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = sample * len(times) / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s32", "data": "synthetic",
+        "config": dict(workload_config(args.had_block), sample=f"{sample} of {TOKENS} token rows against the full W"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"{sample} of {TOKENS} token rows (X rows quantized, W quantized, "
+                                   f"{sample}x{OUT}x{HIDDEN} integer contraction, scale product), per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------ GPU arm
+
+def run_gpu(args, rank: int, world: int, local: int):
+    import numpy as np
+    import torch
+
+    import paper_2502_05003_b200 as quest
+    from paper_2502_05003_b200 import synth
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    g = args.had_block
+    cfg = synth.config2()
+    x_host = torch.from_numpy(cfg["x"]).view(torch.bfloat16).pin_memory()
+    w_host = torch.from_numpy(cfg["w"]).view(torch.bfloat16).pin_memory()
+    M, K, N = TOKENS, HIDDEN, OUT
+    cb = quest.container_bits(BITS)
+
+    def make_set():
+        return {
+            "x": x_host.to(dev), "w": w_host.to(dev),
+            "y": torch.empty((M, N), dtype=torch.bfloat16, device=dev),
+            "saved": {"xq": torch.empty((M, K * cb // 8), dtype=torch.uint8, device=dev),
+                      "sx": torch.empty(M, dtype=torch.float32, device=dev),
+                      "mx": torch.empty((M, K // 8), dtype=torch.uint8, device=dev),
+                      "wq": torch.empty((N, K * cb // 8), dtype=torch.uint8, device=dev),
+                      "sw": torch.empty(N, dtype=torch.float32, device=dev),
+                      "mw": torch.empty((N, K // 8), dtype=torch.uint8, device=dev)},
+            "ws": quest.alloc_workspace(M, N, K, BITS, BITS, dev),
+        }
+
+    one = make_set()
+    set_bytes = sum(t.numel() * t.element_size() for t in [one["x"], one["w"], one["y"], one["ws"]] +
+                    list(one["saved"].values()))
+    n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / set_bytes)))
+    ring = [one] + [make_set() for _ in range(n_sets - 1)]
+
+    def step(i):
+        s = ring[i % n_sets]
+        quest.quest_linear_fwd(s["x"], s["w"], BITS, g, 1.0, y=s["y"], saved=s["saved"], workspace=s["ws"])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------------
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        for i in range(args.steps):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+    elapsed_s = e0.elapsed_time(e1) * 1e-3
+    barrier()
+    status = quest.quest_device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after the timed region")
+    max_elapsed = max_over_ranks(elapsed_s, world, dev)
+    value = aggregate_tokens_per_s(M, args.steps, world, max_elapsed)
+
+    # ---- per-kernel durations: same loop, stages bracketed by CUDA events on the same stream
+    quest.quest_stage_timing(True)
+    quest.quest_stage_times(reset=True)
+    prof_steps = min(args.steps, 200)
+    for i in range(prof_steps):
+        step(i)
+        quest.quest_stage_times()
+    stage = quest.quest_stage_times(reset=True)
+    quest.quest_stage_timing(False)
+    stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+
+    # ---- end to end: pinned host inputs in, result out, every step ---------------------
+    y_host = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    e2e_steps = min(args.steps, 100)
+
+    def e2e_step(i):
+        s = ring[i % n_sets]
+        s["x"].copy_(x_host, non_blocking=True)
+        s["w"].copy_(w_host, non_blocking=True)
+        quest.quest_linear_fwd(s["x"], s["w"], BITS, g, 1.0, y=s["y"], saved=s["saved"], workspace=s["ws"])
+        y_host.copy_(s["y"], non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3, world, dev)
+    e2e_value = aggregate_tokens_per_s(M, e2e_steps, world, e2e_elapsed)
+    h2d = x_host.numel() * 2 + w_host.numel() * 2
+    d2h = y_host.numel() * 2
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    src = "of measured" if peaks["_source"] == "measured" else "of fallback"
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
+    gemm_ms = stage_ms["gemm"]
+    gemm_tops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12 if gemm_ms else None
+    qx_bytes, qw_bytes = quantizer_bytes(M, K, BITS), quantizer_bytes(N, K, BITS)
+    qx_ms, qw_ms = stage_ms["quant_x"], stage_ms["quant_w"]
+    qx_gbs = qx_bytes / (qx_ms * 1e-3) / 1e9 if qx_ms else None
+
+    # int8 library GEMM on the same shape, as a cross-check of the tensor-pipe denominator
+    lib_tops = None
+    try:
+        a8 = torch.randint(-8, 8, (M, K), dtype=torch.int8, device=dev)
+        b8 = torch.randint(-8, 8, (K, N), dtype=torch.int8, device=dev)
+        for _ in range(3):
+            torch._int_mm(a8, b8)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(20):
+            torch._int_mm(a8, b8)
+        e1.record()
+        torch.cuda.synchronize()
+        lib_tops = 2.0 * M * N * K * 20 / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    except Exception:
+        lib_tops = None
+
+    sample = args.ref_tokens if args.ref_tokens > 0 else TOKENS
+    o_dt, o_threads = time_oracle(sample, g)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * max_elapsed / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8",
+        "data": "synthetic",
+        "config": dict(workload_config(g), parallelism=f"replicas x{world}",
+                       l2="ring of %d buffer sets (%.0f MB) larger than L2; no flush" % (n_sets, n_sets * set_bytes / 1e6)),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clocks.summary(),
+        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel (tcgen05 kind::i8)", "achieved": gemm_tops,
+                     "peak": int8_peak, "unit": "TOP/s", "frac": (gemm_tops / int8_peak) if gemm_tops else None,
+                     "peak_basis": f"2 x bf16 burst {src} ({peaks['bf16_tflops']} TFLOP/s)",
+                     "traffic": GEMM_DRAM_TRAFFIC_BYTES, "ms": gemm_ms,
+                     "library_int8_gemm_tops_same_shape": lib_tops},
+        "roofline_quantizer": {"bound": "hbm", "kernel": "quantize (x)", "achieved": qx_gbs,
+                               "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": (qx_gbs / peaks["hbm_gbs"]) if qx_gbs else None, "peak_basis": src,
+                               "traffic": QUANT_DRAM_TRAFFIC_BYTES, "ms": qx_ms,
+                               "algorithmic_bytes": qx_bytes, "w_ms": qw_ms, "w_algorithmic_bytes": qw_bytes},
+        "stage_ms": stage_ms,
+        "cpu_baseline": {"value": sample / o_dt, "unit": UNIT, "cores": o_threads, "kind": "oracle",
+                         "sample": f"{sample} of {TOKENS} token rows against the full W, one pass"},
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="quest", choices=["quest", "reference"])
+    ap.add_argument("--had-block", type=int, default=128)
+    ap.add_argument("--ref-tokens", type=int, default=0,
+                    help="token rows in the CPU oracle's bounded sample (0: the full 4096 for the "
+                         "cpu_baseline leg; sized to about a minute in total for --impl reference)")
+    args = ap.parse_args()
+    rank, world, local = init_ranks(args.gpus)
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_gpu(args, rank, world, local)
+
+
+if __name__ == "__main__":
+    main()

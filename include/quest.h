@@ -1,0 +1,179 @@
+/*
+ * quest.h -- C ABI of the B200 (sm_100a) QuEST quantized-linear forward library.
+ *
+ * The library implements the forward pass of one QuEST linear layer (Algorithm 1 of
+ * "QuEST: Stable Training of LLMs with 1-Bit Weights and Activations", arXiv 2502.05003):
+ *
+ *     x_h = HT(x);  xq_h = proj_{alpha*}(x_h);  w_h = HT(w);  wq_h = proj_{alpha*}(w_h);
+ *     y   = xq_h wq_h^T;   return y, xq_h, wq_h, M(x_h; xq_h), M(w_h; wq_h)
+ *
+ * General rules for every entry point
+ *   - Pointers named in "device" are CUDA device pointers owned by the caller; the library
+ *     allocates no device memory.  Inputs are never written; inputs and outputs must not alias.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and the call returns without synchronising; outputs are valid once the stream reaches
+ *     that point.
+ *   - The return value is a quest_status; 0 is success.  All argument checks run on the host
+ *     before anything is launched: on an argument error nothing is enqueued.  The library
+ *     never throws, aborts or traps.
+ *   - Tensors are row-major.  `dtype`: QUEST_F32 (binary32) or QUEST_BF16 (bfloat16).
+ *
+ * Packed formats (shared by every entry point)
+ *   - Level index k in [0, 2^b - 1]; the grid value is c = 2k - (2^b - 1), an odd integer, and
+ *     the dequantised element is scale[row] * c (Eq. 1's zero-free uniform grid).
+ *   - Codes: container(b) = 1, 2, 4, 4, 8, 8, 8, 8 bits for b = 1..8; a row of `cols` codes
+ *     occupies cols*container/8 bytes, rows are dense; element e of a row sits in byte
+ *     e / (8/container) at bit offset (e mod (8/container)) * container (element 0 lowest).
+ *   - Trust mask: one bit per element, row of cols/8 bytes, element e at bit (e mod 8) of
+ *     byte e/8; 1 = trusted (gradient passes), 0 = masked.
+ *   - Scales: one binary32 per row, the half step of the row's grid in the orthonormal
+ *     Hadamard domain: alpha*(b) * RMS(x_h) / (2^b - 1).
+ */
+#ifndef QUEST_H_
+#define QUEST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum quest_status {
+    QUEST_OK = 0,
+    QUEST_ERR_NULL = 1,           /* a required pointer is NULL */
+    QUEST_ERR_SHAPE = 2,          /* rows/cols/M/N/K/ld out of range or not a supported multiple */
+    QUEST_ERR_BITS = 3,           /* bits outside 1..8 */
+    QUEST_ERR_HAD_BLOCK = 4,      /* had_block not a power of two, does not divide cols, or > 16384 */
+    QUEST_ERR_DTYPE = 5,          /* unknown dtype code */
+    QUEST_ERR_ALIGN = 6,          /* a pointer or leading dimension is not aligned as required */
+    QUEST_ERR_TRUST = 7,          /* trust_factor negative, infinite or NaN */
+    QUEST_ERR_WORKSPACE = 8,      /* workspace NULL or smaller than quest_workspace_bytes() */
+    QUEST_ERR_OVERFLOW = 9,       /* K*(2^bx-1)*(2^bw-1) does not fit in int32 */
+    QUEST_ERR_DEVICE = 10,        /* current device is not compute capability 10.x */
+    QUEST_ERR_CUDA = 11,          /* a CUDA runtime/driver call failed; see quest_last_cuda_error() */
+    QUEST_ERR_DEVICE_TIMEOUT = 12 /* a bounded wait inside a kernel expired (see quest_device_status) */
+} quest_status;
+
+enum { QUEST_F32 = 0, QUEST_BF16 = 1 };
+
+/*
+ * quest_quantize -- lines 2-3 (or 4-5) of Algorithm 1 for every row of x: the Hadamard
+ * rotation of Eq. 2, the RMS normalisation and alpha*(b) clipping of Section 3.1 ("Gaussian
+ * Fitting"), rounding onto Eq. 1's b-bit grid, and the trust mask of Section 3.2.
+ *
+ *   x            device, [rows x cols], row stride ld_elems elements, dtype as given; 16-byte
+ *                aligned, ld_elems*sizeof(elem) a multiple of 16
+ *   rows, cols   rows >= 0 (0 is a no-op); 8 <= cols <= 16384, cols % 8 == 0
+ *   bits         b in 1..8
+ *   had_block    g: the rotation is block-diagonal with the Sylvester-Hadamard matrix H_g on
+ *                contiguous blocks of g elements; a power of two dividing cols (1 = no rotation)
+ *   trust_factor s >= 0: M = [|x_h - xq_h| <= s * alpha* RMS/(2^b-1)] ("The 1-bit Case": s = 1.3
+ *                at b = 1; 1.0 otherwise)
+ *   codes        device out, rows*cols*container/8 bytes, 16-byte aligned; may be NULL
+ *   scales       device out, rows binary32; may be NULL
+ *   mask         device out, rows*cols/8 bytes, 4-byte aligned; may be NULL
+ * Rounding decisions are taken in binary32 in a fixed operation order (descending-stride
+ * butterflies, pairwise sum of squares, one fused multiply-add onto the level axis, ties to
+ * even), so codes and masks are reproducible bit for bit.  A row of zeros gets scale 0, the
+ * middle level and an all-ones mask (for s >= 1).
+ */
+int quest_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
+                   int bits, int had_block, float trust_factor,
+                   uint8_t *codes, float *scales, uint8_t *mask, void *stream);
+
+/*
+ * quest_trust_mask -- the trust mask M_{alpha*}(x_h; xq_h) of Section 3.2 alone (what Algorithm 1
+ * returns for the backward pass), recomputed from x.  Same arguments and rules as
+ * quest_quantize; `mask` is required.
+ */
+int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
+                     int bits, int had_block, float trust_factor, uint8_t *mask, void *stream);
+
+/*
+ * quest_lowbit_gemm -- line 6 of Algorithm 1 on packed codes: acc[i][j] = sum_k cx[i][k]*cw[j][k]
+ * in exact int32 (tensor cores, int8 operands), then y[i][j] = sx[i]*sw[j]*acc[i][j]
+ * (Section 5: integer matmul with the dequantisation fused into the epilogue).
+ *
+ *   xq, sx, bits_x   device: codes [M x K] and scales [M] of the activations
+ *   wq, sw, bits_w   device: codes [N x K] and scales [N] of the weights (both operands K-major)
+ *   M, N, K          M, N >= 0; K >= 32, K % 32 == 0; K*(2^bx-1)*(2^bw-1) < 2^31
+ *   y, y_dtype, ldy  device out [M x N], row stride ldy elements, QUEST_F32 or QUEST_BF16;
+ *                    may be NULL if only acc is wanted
+ *   acc              device out, dense [M x N] int32 raw accumulators; may be NULL
+ *   workspace        device scratch of at least quest_workspace_bytes(M, N, K, bits_x, bits_w)
+ *                    bytes, 256-byte aligned; holds the int8 operands the tensor cores read.
+ *                    Its contents are undefined afterwards; two calls that overlap on the GPU
+ *                    must not share it.
+ */
+int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
+                      const uint8_t *wq, const float *sw, int bits_w,
+                      int64_t M, int64_t N, int64_t K,
+                      void *y, int y_dtype, int64_t ldy_elems, int32_t *acc,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * quest_linear_fwd -- Algorithm 1 end to end: quantize x rows, quantize w rows (unless cached),
+ * contract, scale.  No inverse transform is applied to y: the same rotation on both operands
+ * cancels in the product ("Implementation" paragraph of Section 3.3).
+ *
+ *   x [M x K], w [N x K]   device, dense row-major, `dtype`
+ *   y [M x N]              device out, dense, `y_dtype`
+ *   xq, sx, mx             device out: codes, scales, trust mask of x (Algorithm 1, line 7);
+ *                          xq and sx are required, mx may be NULL
+ *   wq, sw, mw             the same for w.  If w_is_cached != 0, w may be NULL and wq/sw are
+ *                          INPUTS produced by an earlier call with the same bits and had_block
+ *                          (the inference pipeline of Section 5); mw is then untouched
+ *   workspace              as for quest_lowbit_gemm with bits_x = bits_w = bits
+ */
+int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                     int bits, int had_block, float trust_factor,
+                     void *y, int y_dtype,
+                     uint8_t *xq, float *sx, uint8_t *mx,
+                     uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* Bytes of scratch quest_lowbit_gemm / quest_linear_fwd need (0 on invalid arguments). */
+size_t quest_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w);
+
+/* rows*cols*container(bits)/8, the size of a packed code tensor (0 on invalid arguments). */
+size_t quest_codes_bytes(int64_t rows, int64_t cols, int bits);
+
+/* The binary32 table entry alpha*(b) of Section 3.1 (0 outside 1..8). */
+float quest_alpha_star(int bits);
+
+/*
+ * Kernels never spin without bound: a wait that expires records a non-zero word on the device
+ * and the kernel returns.  quest_device_status synchronises `stream`, reads that word, clears
+ * it, and returns QUEST_OK or QUEST_ERR_DEVICE_TIMEOUT (QUEST_ERR_CUDA if the read fails).
+ */
+int quest_device_status(void *stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): per-stage device times.  While enabled, every
+ * entry point brackets each of its stages with a pair of CUDA events on the caller's stream.
+ * quest_stage_times waits for the events of the most recent call, adds their elapsed times to
+ * running totals, copies totals (milliseconds) and counts into the caller's HOST arrays of
+ * QUEST_NUM_STAGES entries (either may be NULL), and zeroes the totals if reset != 0.  Call it
+ * after every timed call: events are reused from call to call.  Not thread-safe; leave it
+ * disabled (the default) in production.
+ */
+enum {
+    QUEST_STAGE_QUANT_X = 0,   /* quantizer launch on x (or the only launch of quest_quantize) */
+    QUEST_STAGE_QUANT_W = 1,   /* quantizer launch on w inside quest_linear_fwd */
+    QUEST_STAGE_UNPACK = 2,    /* packed codes -> int8 operands (and row sums) */
+    QUEST_STAGE_GEMM = 3,      /* the tensor-core contraction with its epilogue */
+    QUEST_NUM_STAGES = 4
+};
+int quest_stage_timing(int enable);
+int quest_stage_times(double *total_ms, long long *counts, int reset);
+
+/* Text for a status code; for QUEST_ERR_CUDA, quest_last_cuda_error() has the CUDA message of
+ * the most recent failure on the calling thread. */
+const char *quest_status_string(int status);
+const char *quest_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QUEST_H_ */

@@ -1,0 +1,182 @@
+"""B200 (sm_100a) implementation of the QuEST quantized-linear forward pass (arXiv 2502.05003,
+Algorithm 1).  This module is a thin binding over the C ABI in ``include/quest.h``: it marshals
+torch tensors (device memory, current stream) into pointers and sizes; every step of the path
+runs in the CUDA library.  There is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+
+import torch
+
+from . import _lib
+from ._lib import QuestError  # noqa: F401
+
+F32, BF16 = 0, 1
+_DT = {torch.float32: F32, torch.bfloat16: BF16}
+
+
+def container_bits(bits: int) -> int:
+    return 1 if bits == 1 else 2 if bits == 2 else 4 if bits <= 4 else 8
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype not in _DT:
+        raise TypeError(f"unsupported dtype {t.dtype}: float32 or bfloat16")
+    return _DT[t.dtype]
+
+
+def _require_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise ValueError("quest: tensors must live in CUDA device memory")
+
+
+def quest_alpha_star(bits: int) -> float:
+    return float(_lib.load().quest_alpha_star(bits))
+
+
+def quest_codes_bytes(rows: int, cols: int, bits: int) -> int:
+    return int(_lib.load().quest_codes_bytes(rows, cols, bits))
+
+
+def quest_workspace_bytes(M: int, N: int, K: int, bits_x: int, bits_w: int) -> int:
+    return int(_lib.load().quest_workspace_bytes(M, N, K, bits_x, bits_w))
+
+
+def quest_device_status() -> int:
+    return int(_lib.load().quest_device_status(_stream()))
+
+
+STAGES = ("quant_x", "quant_w", "unpack", "gemm")
+
+
+def quest_stage_timing(enable: bool) -> None:
+    _lib.check(_lib.load().quest_stage_timing(1 if enable else 0))
+
+
+def quest_stage_times(reset: bool = False) -> dict:
+    """Collects the events of the latest call; returns {stage: (total_ms, count)}."""
+    tot = (ctypes.c_double * len(STAGES))()
+    cnt = (ctypes.c_longlong * len(STAGES))()
+    _lib.check(_lib.load().quest_stage_times(tot, cnt, 1 if reset else 0))
+    return {name: (float(tot[i]), int(cnt[i])) for i, name in enumerate(STAGES)}
+
+
+def alloc_workspace(M: int, N: int, K: int, bits_x: int, bits_w: int, device=None) -> torch.Tensor:
+    n = quest_workspace_bytes(M, N, K, bits_x, bits_w)
+    if n == 0:
+        raise ValueError("quest: invalid GEMM shape or bit-widths")
+    return torch.empty(n, dtype=torch.uint8, device=device or torch.device("cuda"))
+
+
+def quest_quantize(x: torch.Tensor, bits: int, had_block: int, trust_factor: float = 1.0,
+                   codes: torch.Tensor = None, scales: torch.Tensor = None, mask: torch.Tensor = None,
+                   want_mask: bool = True):
+    """Rows of ``x`` [rows, cols] -> (codes uint8 [rows, cols*container/8], scales f32 [rows],
+    mask uint8 [rows, cols/8] or None)."""
+    _require_cuda(x, codes, scales, mask)
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("quest_quantize: x must be 2-D with unit inner stride")
+    rows, cols = x.shape
+    cb = container_bits(bits) if 1 <= bits <= 8 else 8
+    if codes is None:
+        codes = torch.empty((rows, cols * cb // 8), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty(rows, dtype=torch.float32, device=x.device)
+    if mask is None and want_mask:
+        mask = torch.empty((rows, cols // 8), dtype=torch.uint8, device=x.device)
+    st = _lib.load().quest_quantize(_p(x), _dtype_code(x), rows, cols, x.stride(0), bits, had_block,
+                                    ctypes.c_float(trust_factor), _p(codes), _p(scales), _p(mask), _stream())
+    _lib.check(st)
+    return codes, scales, mask
+
+
+def quest_trust_mask(x: torch.Tensor, bits: int, had_block: int, trust_factor: float = 1.0,
+                     mask: torch.Tensor = None) -> torch.Tensor:
+    _require_cuda(x, mask)
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("quest_trust_mask: x must be 2-D with unit inner stride")
+    rows, cols = x.shape
+    if mask is None:
+        mask = torch.empty((rows, cols // 8), dtype=torch.uint8, device=x.device)
+    st = _lib.load().quest_trust_mask(_p(x), _dtype_code(x), rows, cols, x.stride(0), bits, had_block,
+                                      ctypes.c_float(trust_factor), _p(mask), _stream())
+    _lib.check(st)
+    return mask
+
+
+def quest_lowbit_gemm(xq: torch.Tensor, sx: torch.Tensor, bits_x: int,
+                      wq: torch.Tensor, sw: torch.Tensor, bits_w: int, K: int,
+                      out_dtype=torch.bfloat16, y: torch.Tensor = None, want_acc: bool = False,
+                      acc: torch.Tensor = None, workspace: torch.Tensor = None, want_y: bool = True):
+    """Packed codes -> (y [M, N] or None, acc int32 [M, N] or None)."""
+    _require_cuda(xq, sx, wq, sw, y, acc, workspace)
+    M, N = xq.shape[0], wq.shape[0]
+    if y is None and want_y:
+        y = torch.empty((M, N), dtype=out_dtype, device=xq.device)
+    if acc is None and want_acc:
+        acc = torch.empty((M, N), dtype=torch.int32, device=xq.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, bits_x, bits_w, xq.device)
+    st = _lib.load().quest_lowbit_gemm(_p(xq), _p(sx), bits_x, _p(wq), _p(sw), bits_w, M, N, K,
+                                       _p(y), _dtype_code(y) if y is not None else 0,
+                                       y.stride(0) if y is not None else N, _p(acc),
+                                       _p(workspace), workspace.numel(), _stream())
+    _lib.check(st)
+    return y, acc
+
+
+def quest_linear_fwd(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int, trust_factor: float = 1.0,
+                     out_dtype=None, y: torch.Tensor = None, saved: dict = None, w_cached: dict = None,
+                     workspace: torch.Tensor = None, want_masks: bool = True) -> dict:
+    """Algorithm 1: returns {"y", "xq", "sx", "mx", "wq", "sw", "mw"}.
+
+    ``saved`` may carry preallocated output tensors under those keys; ``w_cached`` = {"wq", "sw"}
+    from an earlier call skips the weight quantization (then ``w`` may be None).
+    """
+    _require_cuda(x, w, y, workspace)
+    M, K = x.shape
+    out = dict(saved or {})
+    if w_cached is not None:
+        out["wq"], out["sw"] = w_cached["wq"], w_cached["sw"]
+        N = out["wq"].shape[0]
+    else:
+        N = w.shape[0]
+    cb = container_bits(bits) if 1 <= bits <= 8 else 8
+    dev = x.device
+
+    def need(key, shape, dtype):
+        if out.get(key) is None:
+            out[key] = torch.empty(shape, dtype=dtype, device=dev)
+
+    need("xq", (M, K * cb // 8), torch.uint8)
+    need("sx", (M,), torch.float32)
+    need("wq", (N, K * cb // 8), torch.uint8)
+    need("sw", (N,), torch.float32)
+    if want_masks:
+        need("mx", (M, K // 8), torch.uint8)
+        if w_cached is None:
+            need("mw", (N, K // 8), torch.uint8)
+    out.setdefault("mx", None)
+    out.setdefault("mw", None)
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, bits, bits, dev)
+    st = _lib.load().quest_linear_fwd(
+        _p(x), _p(w), _dtype_code(x), M, N, K, bits, had_block, ctypes.c_float(trust_factor),
+        _p(y), _dtype_code(y), _p(out["xq"]), _p(out["sx"]), _p(out["mx"]),
+        _p(out["wq"]), _p(out["sw"]), _p(out["mw"]), 1 if w_cached is not None else 0,
+        _p(workspace), workspace.numel(), _stream())
+    _lib.check(st)
+    out["y"] = y
+    return out

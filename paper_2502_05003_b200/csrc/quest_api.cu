@@ -1,0 +1,297 @@
+// extern "C" entry points of the library: host-side argument validation, workspace carving and
+// the launch sequence of each call.  Declarations and argument documentation: include/quest.h.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "quest_internal.cuh"
+
+namespace quest {
+
+// Written by a kernel whose bounded wait expired; read and cleared by quest_device_status.
+__device__ int g_timeout_word = 0;
+
+static thread_local char t_cuda_msg[256] = "";
+
+int cuda_fail(cudaError_t e) {
+    snprintf(t_cuda_msg, sizeof(t_cuda_msg), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return QUEST_ERR_CUDA;
+}
+int cuda_fail_msg(const char *msg) {
+    snprintf(t_cuda_msg, sizeof(t_cuda_msg), "%s", msg);
+    return QUEST_ERR_CUDA;
+}
+
+int *device_status_word() {
+    static int *cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_timeout_word);
+        if (e != cudaSuccess) {
+            cuda_fail(e);
+            return nullptr;
+        }
+        cached[dev] = reinterpret_cast<int *>(p);
+    }
+    return cached[dev];
+}
+
+int check_device() {
+    static int cached[64] = {0};   // 0 unknown, 1 ok, 2 wrong architecture
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return QUEST_ERR_DEVICE;
+    if (!cached[dev]) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        cached[dev] = (major == 10) ? 1 : 2;
+    }
+    return cached[dev] == 1 ? QUEST_OK : QUEST_ERR_DEVICE;
+}
+
+// Optional per-stage timing: CUDA events recorded on the caller's stream around each stage.
+struct StageTimer {
+    bool enabled = false;
+    cudaEvent_t ev[QUEST_NUM_STAGES][2] = {};
+    bool created = false;
+    bool pending[QUEST_NUM_STAGES] = {};
+    double total_ms[QUEST_NUM_STAGES] = {};
+    long long count[QUEST_NUM_STAGES] = {};
+};
+static StageTimer g_timer;
+
+struct StageScope {
+    int id;
+    cudaStream_t st;
+    bool on;
+    StageScope(int id_, cudaStream_t st_) : id(id_), st(st_), on(g_timer.enabled && g_timer.created) {
+        if (on) cudaEventRecord(g_timer.ev[id][0], st);
+    }
+    ~StageScope() {
+        if (on) {
+            cudaEventRecord(g_timer.ev[id][1], st);
+            g_timer.pending[id] = true;
+        }
+    }
+};
+
+static bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+static bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static int validate_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld, int bits,
+                             int had_block, float trust_factor, const uint8_t *codes, const uint8_t *mask) {
+    if (!x && rows != 0) return QUEST_ERR_NULL;
+    if (dtype != QUEST_F32 && dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+    if (bits < 1 || bits > 8) return QUEST_ERR_BITS;
+    if (rows < 0 || rows > (int64_t)1 << 31 || cols < 8 || cols > 16384 || cols % 8 != 0 || ld < cols)
+        return QUEST_ERR_SHAPE;
+    if (!is_pow2(had_block) || had_block > cols || cols % had_block != 0) return QUEST_ERR_HAD_BLOCK;
+    if (!(trust_factor >= 0.0f) || isinf(trust_factor)) return QUEST_ERR_TRUST;
+    const size_t esz = dtype == QUEST_F32 ? 4 : 2;
+    if (!aligned(x, 16) || (ld * esz) % 16 != 0) return QUEST_ERR_ALIGN;
+    if (codes && !aligned(codes, 16)) return QUEST_ERR_ALIGN;
+    if (mask && !aligned(mask, 4)) return QUEST_ERR_ALIGN;
+    return QUEST_OK;
+}
+
+static int validate_gemm_shape(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w) {
+    if (bits_x < 1 || bits_x > 8 || bits_w < 1 || bits_w > 8) return QUEST_ERR_BITS;
+    if (M < 0 || N < 0 || M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K < 32 || K % 32 != 0 ||
+        K > (int64_t)1 << 24)
+        return QUEST_ERR_SHAPE;
+    const int64_t worst = K * (((int64_t)1 << bits_x) - 1) * (((int64_t)1 << bits_w) - 1);
+    if (worst >= ((int64_t)1 << 31)) return QUEST_ERR_OVERFLOW;
+    return QUEST_OK;
+}
+
+}  // namespace quest
+
+using namespace quest;
+
+extern "C" {
+
+float quest_alpha_star(int bits) { return alpha_star(bits); }
+
+size_t quest_codes_bytes(int64_t rows, int64_t cols, int bits) {
+    if (rows < 0 || cols < 0 || bits < 1 || bits > 8) return 0;
+    return (size_t)rows * (size_t)cols * (size_t)container_bits(bits) / 8;
+}
+
+size_t quest_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w) {
+    if (validate_gemm_shape(M, N, K, bits_x, bits_w) != QUEST_OK) return 0;
+    size_t b = carve_workspace(nullptr, M, N, K).bytes;
+    return b ? b : 256;
+}
+
+const char *quest_status_string(int status) {
+    switch (status) {
+        case QUEST_OK: return "ok";
+        case QUEST_ERR_NULL: return "a required pointer is NULL";
+        case QUEST_ERR_SHAPE: return "unsupported shape or leading dimension";
+        case QUEST_ERR_BITS: return "bits must be in 1..8";
+        case QUEST_ERR_HAD_BLOCK: return "had_block must be a power of two that divides cols";
+        case QUEST_ERR_DTYPE: return "unknown dtype code";
+        case QUEST_ERR_ALIGN: return "pointer or leading dimension not aligned as required";
+        case QUEST_ERR_TRUST: return "trust_factor must be finite and >= 0";
+        case QUEST_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case QUEST_ERR_OVERFLOW: return "K*(2^bx-1)*(2^bw-1) does not fit in int32";
+        case QUEST_ERR_DEVICE: return "current device is not compute capability 10.x";
+        case QUEST_ERR_CUDA: return "CUDA call failed";
+        case QUEST_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        default: return "unknown status";
+    }
+}
+
+const char *quest_last_cuda_error(void) { return t_cuda_msg; }
+
+int quest_device_status(void *stream) {
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int *word = device_status_word();
+    if (!word) return QUEST_ERR_CUDA;
+    int v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, word, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (v != 0) {
+        e = cudaMemsetAsync(word, 0, sizeof(int), st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        return QUEST_ERR_DEVICE_TIMEOUT;
+    }
+    return QUEST_OK;
+}
+
+int quest_stage_timing(int enable) {
+    if (enable && !g_timer.created) {
+        for (int i = 0; i < QUEST_NUM_STAGES; ++i)
+            for (int j = 0; j < 2; ++j) {
+                cudaError_t e = cudaEventCreate(&g_timer.ev[i][j]);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
+        g_timer.created = true;
+    }
+    g_timer.enabled = enable != 0;
+    return QUEST_OK;
+}
+
+int quest_stage_times(double *total_ms, long long *counts, int reset) {
+    for (int i = 0; i < QUEST_NUM_STAGES; ++i) {
+        if (g_timer.pending[i]) {
+            cudaError_t e = cudaEventSynchronize(g_timer.ev[i][1]);
+            float ms = 0.0f;
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, g_timer.ev[i][0], g_timer.ev[i][1]);
+            if (e != cudaSuccess) return cuda_fail(e);
+            g_timer.total_ms[i] += ms;
+            g_timer.count[i] += 1;
+            g_timer.pending[i] = false;
+        }
+        if (total_ms) total_ms[i] = g_timer.total_ms[i];
+        if (counts) counts[i] = g_timer.count[i];
+        if (reset) {
+            g_timer.total_ms[i] = 0.0;
+            g_timer.count[i] = 0;
+        }
+    }
+    return QUEST_OK;
+}
+
+int quest_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
+                   int bits, int had_block, float trust_factor,
+                   uint8_t *codes, float *scales, uint8_t *mask, void *stream) {
+    int s = validate_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, codes, mask);
+    if (s) return s;
+    if ((s = check_device())) return s;
+    StageScope scope(QUEST_STAGE_QUANT_X, reinterpret_cast<cudaStream_t>(stream));
+    return launch_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, codes, scales, mask,
+                           nullptr, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
+                     int bits, int had_block, float trust_factor, uint8_t *mask, void *stream) {
+    if (!mask) return QUEST_ERR_NULL;
+    int s = validate_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, nullptr, mask);
+    if (s) return s;
+    if ((s = check_device())) return s;
+    return launch_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, nullptr, nullptr, mask,
+                           nullptr, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
+                      const uint8_t *wq, const float *sw, int bits_w,
+                      int64_t M, int64_t N, int64_t K,
+                      void *y, int y_dtype, int64_t ldy_elems, int32_t *acc,
+                      void *workspace, size_t workspace_bytes, void *stream) {
+    int s = validate_gemm_shape(M, N, K, bits_x, bits_w);
+    if (s) return s;
+    if (M == 0 || N == 0) return QUEST_OK;            /* empty product: nothing to write */
+    if (!xq || !wq) return QUEST_ERR_NULL;
+    if (!y && !acc) return QUEST_ERR_NULL;
+    if (y && (!sx || !sw)) return QUEST_ERR_NULL;
+    if (y) {
+        if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+        if (ldy_elems < N) return QUEST_ERR_SHAPE;
+        if (!aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    }
+    if (!aligned(xq, 16) || !aligned(wq, 16) || (acc && !aligned(acc, 4))) return QUEST_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, bits_x, bits_w))
+        return QUEST_ERR_WORKSPACE;
+    if ((s = check_device())) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    Workspace ws = carve_workspace(workspace, M, N, K);
+    const bool need_rs_a = bits_w == 8;    // sum of x operand values multiplies the offset of the w codes
+    const bool need_rs_b = bits_x == 8;
+    {
+        StageScope scope(QUEST_STAGE_UNPACK, st);
+        if ((s = launch_unpack(xq, bits_x, M, K, ws.a8, need_rs_a ? ws.rs_a : nullptr, st))) return s;
+        if ((s = launch_unpack(wq, bits_w, N, K, ws.b8, need_rs_b ? ws.rs_b : nullptr, st))) return s;
+    }
+    StageScope scope(QUEST_STAGE_GEMM, st);
+    return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits_x, bits_w, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc,
+                       st);
+}
+
+int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                     int bits, int had_block, float trust_factor,
+                     void *y, int y_dtype,
+                     uint8_t *xq, float *sx, uint8_t *mx,
+                     uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                     void *workspace, size_t workspace_bytes, void *stream) {
+    if (!y || !xq || !sx || !wq || !sw) return QUEST_ERR_NULL;
+    if (!w_is_cached && !w) return QUEST_ERR_NULL;
+    if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+    int s = validate_gemm_shape(M, N, K, bits, bits);
+    if (s) return s;
+    if ((s = validate_quantize(x, dtype, M, K, K, bits, had_block, trust_factor, xq, mx))) return s;
+    if (!w_is_cached && (s = validate_quantize(w, dtype, N, K, K, bits, had_block, trust_factor, wq, mw))) return s;
+    if (!aligned(wq, 16) || !aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, bits, bits))
+        return QUEST_ERR_WORKSPACE;
+    if ((s = check_device())) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    Workspace ws = carve_workspace(workspace, M, N, K);
+    const bool need_rs = bits == 8;
+    // activations: codes, scale, mask and the int8 operand in one pass
+    {
+        StageScope scope(QUEST_STAGE_QUANT_X, st);
+        if ((s = launch_quantize(x, dtype, M, K, K, bits, had_block, trust_factor, xq, sx, mx, ws.a8, st))) return s;
+    }
+    if (w_is_cached) {
+        StageScope scope(QUEST_STAGE_UNPACK, st);
+        if ((s = launch_unpack(wq, bits, N, K, ws.b8, need_rs ? ws.rs_b : nullptr, st))) return s;
+    } else {
+        StageScope scope(QUEST_STAGE_QUANT_W, st);
+        if ((s = launch_quantize(w, dtype, N, K, K, bits, had_block, trust_factor, wq, sw, mw, ws.b8, st))) return s;
+    }
+    if (need_rs) {
+        if ((s = launch_rowsum(ws.a8, M, K, ws.rs_a, st))) return s;
+        if (!w_is_cached && (s = launch_rowsum(ws.b8, N, K, ws.rs_b, st))) return s;
+    }
+    StageScope scope(QUEST_STAGE_GEMM, st);
+    return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits, bits, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);
+}
+
+}  // extern "C"

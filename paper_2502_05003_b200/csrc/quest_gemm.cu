@@ -1,0 +1,532 @@
+// Low-bit GEMM of the QuEST forward pass (Algorithm 1, line 6; Section 5, stage 3) for sm_100a.
+//
+//   acc[i][j] = sum_k cx[i][k] * cw[j][k]   exact int32, 5th-generation tensor cores
+//   y[i][j]   = sx[i] * sw[j] * acc[i][j]   fused into the epilogue, bf16 or fp32 out
+//
+// B200 has no dense 4-bit integer MMA, so the contraction runs as tcgen05.mma kind::i8 on int8
+// operand values held in a caller-provided workspace (written either by the quantizer itself or
+// by unpack_codes_kernel below).  For b < 8 the operand value is the grid value c = 2k-(2^b-1);
+// for b = 8 (|c| up to 255) it is v = k - 128 and the epilogue restores
+// c_x . c_w = 4 v_x.v_w + 2 sum(v_x) + 2 sum(v_w) + K exactly from per-row sums.
+//
+// Kernel structure (one CTA per SM, persistent over 128 x BN output tiles):
+//   warp 0      TMA producer: 128B-swizzled K-major tiles of A (128 x 128 B) and B (BN x 128 B)
+//               into a 4-stage shared-memory ring, completion on mbarriers
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=32) x 4 per stage into
+//               one of two TMEM accumulator buffers; tcgen05.commit releases the stage / signals
+//               the epilogue
+//   warps 2..5  epilogue: tcgen05.ld 32 columns at a time, integer correction, scale, convert,
+//               store; overlaps the next tile's main loop through the second TMEM buffer
+// Every wait is bounded: on expiry the CTA records a status word, stops issuing work and exits
+// through the common tail (which frees its TMEM).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "quest_internal.cuh"
+
+namespace quest {
+namespace {
+
+constexpr int BM = 128;          // tile rows (TMEM lanes)
+constexpr int BK = 128;          // bytes (= int8 elements) of K per pipeline stage: one swizzle row
+constexpr int UMMA_K = 32;       // K per tcgen05.mma kind::i8
+constexpr int STAGES = 4;
+constexpr int NUM_THREADS = 192;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
+
+enum { ST_OK = 0, ST_PRODUCER = 1, ST_MMA = 2, ST_EPILOGUE = 3 };
+
+struct GemmParams {
+    int M, N, K;
+    const float *sx;
+    const float *sw;
+    const int32_t *rs_a;   // row sums of the A operand values (nullable)
+    const int32_t *rs_b;   // row sums of the B operand values (nullable)
+    int mul;               // acc' = mul*acc + ca*rs_a[i] + cb*rs_b[j] + ck
+    int ca, cb, ck;
+    void *y;
+    int y_dtype;
+    long long ldy;
+    int32_t *acc;
+    int *status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting or the limit expired (then it records
+// `code` in the device status word and raises the CTA-wide abort flag).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                       int *status, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 0; it < 0x7fffffffu; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 15u) == 15u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(status, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);          // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                                // leading byte offset (unused with swizzle), bits [16,30)
+    d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                                // descriptor version (sm_100), bits [46,48)
+    d |= (uint64_t)2 << 61;                                // layout: SWIZZLE_128B, bits [61,64)
+    return d;
+}
+// Instruction descriptor for kind::i8: D = s32, A = B = signed 8-bit, both K-major.
+__host__ __device__ constexpr uint32_t make_idesc_i8(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+template <int BN>
+struct SmemLayout {
+    static constexpr int A_BYTES = BM * BK;
+    static constexpr int B_BYTES = BN * BK;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + slack for 1024-byte alignment
+};
+
+template <int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+    using L = SmemLayout<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET);
+    uint64_t *full_bar = bars;                   // [STAGES] TMA -> MMA
+    uint64_t *empty_bar = bars + STAGES;         // [STAGES] MMA -> TMA
+    uint64_t *tfull_bar = bars + 2 * STAGES;     // [2] MMA -> epilogue
+    uint64_t *tempty_bar = bars + 2 * STAGES + 2;  // [2] epilogue -> MMA
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    constexpr uint32_t TMEM_COLS = 2 * BN;       // two accumulator buffers
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tfull_bar[b]), 1);
+            mbar_init(smem_u32(&tempty_bar[b]), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int num_m = (p.M + BM - 1) / BM;
+    const int num_n = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = (p.K + BK - 1) / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % num_m) * BM;
+                const int n0 = (tile / num_m) * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, p.status, ST_PRODUCER);
+                    if (!ok) break;
+                    const uint32_t fb = smem_u32(&full_bar[stage]);
+                    mbar_expect_tx(fb, L::STAGE_BYTES);
+                    uint8_t *sa = smem + stage * L::STAGE_BYTES;
+                    tma_load_2d(smem_u32(sa), &tmA, kb * BK, m0, fb);
+                    tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // aborting: let copies that are still in flight land before the CTA retires
+                for (int s = 0; s < STAGES; ++s) {
+                    const long long t0 = clock64();
+                    while (clock64() - t0 < 200000) { /* bounded drain window */ }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int t = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+                const int buf = t & 1;
+                const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
+                ok = mbar_wait(smem_u32(&tempty_bar[buf]), bphase ^ 1u, abort_flag, p.status, ST_MMA);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_flag, p.status, ST_MMA);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + stage * L::STAGE_BYTES);
+                    const uint64_t a_desc = make_smem_desc(sa);
+                    const uint64_t b_desc = make_smem_desc(sa + L::A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                        // advance along K inside the 128-byte swizzle row: +32 bytes = +2 in 16-byte units
+                        umma_i8(d_tmem, a_desc + (uint64_t)(kk * (UMMA_K >> 4)), b_desc + (uint64_t)(kk * (UMMA_K >> 4)),
+                                idesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&empty_bar[stage]));     // stage reusable once these MMAs retire
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(smem_u32(&tfull_bar[buf]));   // accumulator complete
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quarter = warp & 3;                  // TMEM lane quarter this warp may read
+        int t = 0;
+        bool ok = true;
+        const bool vec_ok_bf16 = p.y && p.y_dtype == QUEST_BF16 && (p.ldy % 8 == 0) &&
+                                 ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const bool vec_ok_f32 = p.y && p.y_dtype == QUEST_F32 && (p.ldy % 4 == 0) &&
+                                ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const bool vec_ok_acc = p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+            const int m0 = (tile % num_m) * BM;
+            const int n0 = (tile / num_m) * BN;
+            const int buf = t & 1;
+            const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
+            ok = mbar_wait(smem_u32(&tfull_bar[buf]), bphase, abort_flag, p.status, ST_EPILOGUE);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int row = m0 + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+            const float sxr = row_ok ? __ldg(p.sx + row) : 0.0f;
+            const int rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (n0 + c0 >= p.N) break;             // uniform across the warp
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + c0), r);
+                if (!row_ok) continue;
+                const int col0 = n0 + c0;
+                int32_t v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    int32_t a = p.mul * (int32_t)r[j] + rsa;
+                    if (p.rs_b && col0 + j < p.N) a += p.cb * __ldg(p.rs_b + col0 + j);
+                    v[j] = a;
+                }
+                if (p.acc) {
+                    int32_t *dst = p.acc + (long long)row * p.N + col0;
+                    if (vec_ok_acc && col0 + 32 <= p.N) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<int4 *>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+                        for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = v[j];
+                    }
+                }
+                if (p.y) {
+                    float f[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float swj = (col0 + j < p.N) ? __ldg(p.sw + col0 + j) : 0.0f;
+                        f[j] = __fmul_rn(__fmul_rn(sxr, swj), (float)v[j]);
+                    }
+                    if (p.y_dtype == QUEST_BF16) {
+                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.y) + (long long)row * p.ldy + col0;
+                        if (vec_ok_bf16 && col0 + 32 <= p.N) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[j], f[j + 1]);
+                                __nv_bfloat162 h1 = __floats2bfloat162_rn(f[j + 2], f[j + 3]);
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[j + 4], f[j + 5]);
+                                __nv_bfloat162 h3 = __floats2bfloat162_rn(f[j + 6], f[j + 7]);
+                                uint4 q;
+                                q.x = *reinterpret_cast<uint32_t *>(&h0);
+                                q.y = *reinterpret_cast<uint32_t *>(&h1);
+                                q.z = *reinterpret_cast<uint32_t *>(&h2);
+                                q.w = *reinterpret_cast<uint32_t *>(&h3);
+                                *reinterpret_cast<uint4 *>(dst + j) = q;
+                            }
+                        } else {
+                            for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
+                        }
+                    } else {
+                        float *dst = reinterpret_cast<float *>(p.y) + (long long)row * p.ldy + col0;
+                        if (vec_ok_f32 && col0 + 32 <= p.N) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4 *>(dst + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+                        } else {
+                            for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = f[j];
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Packed codes -> int8 operand values (and row sums for 8-bit codes).
+// One thread converts 32 consecutive elements (rows are dense and K % 32 == 0).
+// ---------------------------------------------------------------------------------------------
+__global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits, long long n_groups,
+                                    int8_t *__restrict__ out) {
+    const int cb = container_bits(bits);
+    const int L1 = (1 << bits) - 1;
+    const int words = cb;                                   // 32 elements * cb bits = cb 32-bit words
+    for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n_groups;
+         g += (long long)gridDim.x * blockDim.x) {
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(codes) + g * words;
+        uint32_t w[8];
+        for (int i = 0; i < words; ++i) w[i] = __ldg(src + i);
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t packed = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int e = q * 4 + j;
+                const int bitpos = e * cb;
+                const int k = (w[bitpos >> 5] >> (bitpos & 31)) & ((1 << cb) - 1);
+                const int v = (bits == 8) ? (k - 128) : (2 * k - L1);
+                packed |= (uint32_t)(uint8_t)(int8_t)v << (8 * j);
+            }
+            o[q] = packed;
+        }
+        uint4 *dst = reinterpret_cast<uint4 *>(out + g * 32);
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
+// Row sums of an int8 matrix [rows x K]: one warp per row.
+__global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, int K, int32_t *__restrict__ out) {
+    const long long row = blockIdx.x * (long long)(blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const int8_t *r = a + row * (long long)K;
+    int s = 0;
+    for (int k = lane * 4; k < K; k += 128) {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(r + k);
+        s += (int8_t)(w & 0xff) + (int8_t)((w >> 8) & 0xff) + (int8_t)((w >> 16) & 0xff) + (int8_t)(w >> 24);
+    }
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) out[row] = s;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// int8 matrix [rows x K], K contiguous; box = 128 bytes of K x box_rows rows, 128-byte swizzle.
+int make_operand_map(CUtensorMap *tm, const int8_t *base, int64_t rows, int64_t K, int box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return cuda_fail_msg("cuTensorMapEncodeTiled entry point not available");
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail_msg("cuTensorMapEncodeTiled failed");
+    return QUEST_OK;
+}
+
+template <int BN>
+int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SmemLayout<BN>::TOTAL);
+        if (e != cudaSuccess) return cuda_fail(e);
+        attr_done = true;
+    }
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
+    const int grid = tiles < sms ? tiles : sms;
+    gemm_i8_kernel<BN><<<grid, NUM_THREADS, SmemLayout<BN>::TOTAL, st>>>(tmA, tmB, p);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+Workspace carve_workspace(void *base, int64_t M, int64_t N, int64_t K) {
+    Workspace w;
+    size_t off = 0;
+    uint8_t *b = reinterpret_cast<uint8_t *>(base);
+    w.a8 = reinterpret_cast<int8_t *>(b + off);
+    off += align_up((size_t)(M * K), 256);
+    w.b8 = reinterpret_cast<int8_t *>(b + off);
+    off += align_up((size_t)(N * K), 256);
+    w.rs_a = reinterpret_cast<int32_t *>(b + off);
+    off += align_up((size_t)M * 4, 256);
+    w.rs_b = reinterpret_cast<int32_t *>(b + off);
+    off += align_up((size_t)N * 4, 256);
+    w.bytes = off;
+    return w;
+}
+
+int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out, int32_t *rowsum,
+                  cudaStream_t st) {
+    if (rows == 0) return QUEST_OK;
+    const long long n_groups = rows * K / 32;
+    const int threads = 256;
+    long long blocks = (n_groups + threads - 1) / threads;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    unpack_codes_kernel<<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (rowsum) return launch_rowsum(out, rows, K, rowsum, st);
+    return QUEST_OK;
+}
+
+int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st) {
+    if (rows == 0) return QUEST_OK;
+    const long long rb = (rows + 7) / 8;
+    rowsum_i8_kernel<<<(int)rb, 256, 0, st>>>(a8, rows, (int)K, rowsum);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+}
+
+int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
+                int bits_x, int bits_w, const float *sx, const float *sw,
+                int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
+                int32_t *acc, cudaStream_t st) {
+    if (M == 0 || N == 0) return QUEST_OK;
+    // operand value v relates to the grid value c by c = m*v + a: (1, 0) below 8 bits, (2, 1) at 8 bits
+    const int mx = bits_x == 8 ? 2 : 1, ax = bits_x == 8 ? 1 : 0;
+    const int mw = bits_w == 8 ? 2 : 1, aw = bits_w == 8 ? 1 : 0;
+    GemmParams p;
+    p.M = (int)M; p.N = (int)N; p.K = (int)K;
+    p.sx = sx; p.sw = sw;
+    p.mul = mx * mw;
+    p.ca = mx * aw;                        // multiplies sum_k v_x[i][k]
+    p.cb = ax * mw;                        // multiplies sum_k v_w[j][k]
+    p.ck = ax * aw * (int)K;
+    p.rs_a = p.ca ? rs_a : nullptr;
+    p.rs_b = p.cb ? rs_b : nullptr;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc;
+    p.status = device_status_word();
+    if (!p.status) return QUEST_ERR_CUDA;
+
+    const bool wide = N > 128;
+    CUtensorMap tmA, tmB;
+    int s = make_operand_map(&tmA, a8, M, K, BM);
+    if (s) return s;
+    s = make_operand_map(&tmB, b8, N, K, wide ? 256 : 128);
+    if (s) return s;
+    return wide ? launch_gemm_bn<256>(tmA, tmB, p, st) : launch_gemm_bn<128>(tmA, tmB, p, st);
+}
+
+}  // namespace quest

@@ -1,0 +1,71 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "quest.h"
+
+namespace quest {
+
+// alpha*(b), b = 1..8 (Section 3.1): minimiser of the Gaussian quantisation MSE on the
+// 2^b-point grid, rounded to binary32.
+__host__ __device__ inline float alpha_star(int bits) {
+    switch (bits) {
+        case 1: return 0.7978846f;
+        case 2: return 1.4935300f;
+        case 3: return 2.0510680f;
+        case 4: return 2.5140045f;
+        case 5: return 2.9161513f;
+        case 6: return 3.2779846f;
+        case 7: return 3.6110970f;
+        case 8: return 3.9222038f;
+        default: return 0.0f;
+    }
+}
+
+__host__ __device__ inline int container_bits(int bits) {
+    return bits == 1 ? 1 : bits == 2 ? 2 : bits <= 4 ? 4 : 8;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Per-row constants of the projection, computed once on the host in binary32.
+struct QuantConsts {
+    float c0;      // (2^b-1)/2: centre of the level axis
+    float top;     // 2^b-1: highest level
+    float A;       // (2^b-1)/(2 alpha*): RMS-normalised value -> level-axis slope
+    float B;       // alpha*/((2^b-1) sqrt(g)): RMS of the un-normalised rotation -> scale
+    float h;       // trust_factor/2: trust bound in level steps
+};
+QuantConsts make_quant_consts(int bits, int had_block, float trust_factor);
+
+// Operand layout of the int8 tensor-core contraction inside the workspace.
+struct Workspace {
+    int8_t *a8;        // [M x K] int8 operand values of x
+    int8_t *b8;        // [N x K] int8 operand values of w
+    int32_t *rs_a;     // [M] row sums of a8 (used only with 8-bit codes)
+    int32_t *rs_b;     // [N]
+    size_t bytes;
+};
+Workspace carve_workspace(void *base, int64_t M, int64_t N, int64_t K);
+
+// Status / error plumbing.
+int cuda_fail(cudaError_t e);             // records the message, returns QUEST_ERR_CUDA
+int cuda_fail_msg(const char *msg);
+int *device_status_word();                // device address of the timeout word (current device)
+int check_device();                       // QUEST_OK iff current device is sm_10x
+
+// Launchers (each returns a quest_status; arguments already validated).
+int launch_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                    int bits, int had_block, float trust_factor,
+                    uint8_t *codes, float *scales, uint8_t *mask, int8_t *op8, cudaStream_t st);
+int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out,
+                  int32_t *rowsum, cudaStream_t st);
+int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st);
+int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
+                int bits_x, int bits_w, const float *sx, const float *sw,
+                int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
+                int32_t *acc, cudaStream_t st);
+
+}  // namespace quest
