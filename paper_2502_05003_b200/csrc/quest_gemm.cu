@@ -150,10 +150,12 @@ struct SmemLayout {
     static constexpr int B_BYTES = BN * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-    static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + slack for 1024-byte alignment
+    static constexpr int SW_OFFSET = BAR_OFFSET + 256;       // [2][BN] column scales
+    static constexpr int CB_OFFSET = SW_OFFSET + 2 * BN * 4; // [2][BN] column corrections (8-bit codes)
+    static constexpr int TOTAL = CB_OFFSET + 2 * BN * 4 + 1024;   // + slack for 1024-byte alignment
 };
 
-template <int BN>
+template <int BN, bool CORR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
     using L = SmemLayout<BN>;
@@ -166,6 +168,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint64_t *tempty_bar = bars + 2 * STAGES + 2;  // [2] epilogue -> MMA
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    float *sw_tile = reinterpret_cast<float *>(smem + L::SW_OFFSET);
+    int32_t *cb_tile = reinterpret_cast<int32_t *>(smem + L::CB_OFFSET);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -262,85 +266,113 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         __syncwarp();
     } else {
-        const int quarter = warp & 3;                  // TMEM lane quarter this warp may read
+        // ---- epilogue: 4 warps, warp q reads TMEM lanes [32q, 32q+32) = tile rows 32q + lane ----
+        const int quarter = warp & 3;
+        const int ep_tid = threadIdx.x - 64;           // 0..127 over the epilogue warps
         int t = 0;
         bool ok = true;
-        const bool vec_ok_bf16 = p.y && p.y_dtype == QUEST_BF16 && (p.ldy % 8 == 0) &&
-                                 ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
-        const bool vec_ok_f32 = p.y && p.y_dtype == QUEST_F32 && (p.ldy % 4 == 0) &&
-                                ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
-        const bool vec_ok_acc = p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
+        const bool vec_y = p.y && (((reinterpret_cast<uintptr_t>(p.y) & 15) == 0) &&
+                                   (p.ldy % (p.y_dtype == QUEST_BF16 ? 8 : 4) == 0));
+        const bool vec_acc = p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
             const int m0 = (tile % num_m) * BM;
             const int n0 = (tile / num_m) * BN;
             const int buf = t & 1;
             const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
+            // stage this tile's column scales (and column corrections) in shared memory; the
+            // buffer of tile t was last read during tile t-2, which every warp left before it
+            // arrived at the barrier of tile t-1
+            float *swt = sw_tile + buf * BN;
+            int32_t *cbt = cb_tile + buf * BN;
+            for (int c = ep_tid; c < BN; c += 128) {
+                const int col = n0 + c;
+                swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
+                if (CORR) cbt[c] = (p.rs_b && col < p.N) ? p.cb * __ldg(p.rs_b + col) : 0;
+            }
             ok = mbar_wait(smem_u32(&tfull_bar[buf]), bphase, abort_flag, p.status, ST_EPILOGUE);
-            ok = __all_sync(0xffffffffu, ok);
+            // one barrier over the 128 epilogue threads publishes the staged scales and makes the
+            // continue/abort decision unanimous, so no warp can be left waiting at a later barrier
+            {
+                uint32_t all_ok;
+                asm volatile(
+                    "{\n\t.reg .pred p, q;\n\t"
+                    "setp.ne.u32 q, %1, 0;\n\t"
+                    "bar.red.and.pred p, 1, 128, q;\n\t"
+                    "selp.u32 %0, 1, 0, p;\n\t}"
+                    : "=r"(all_ok)
+                    : "r"((uint32_t)(ok ? 1u : 0u))
+                    : "memory");
+                ok = all_ok != 0;
+            }
             if (!ok) break;
             tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
             const bool row_ok = row < p.M;
-            const float sxr = row_ok ? __ldg(p.sx + row) : 0.0f;
-            const int rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
+            const float sxr = (row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
+            int rsa = 0;
+            if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= p.N) break;             // uniform across the warp
+                if (n0 + c0 >= p.N) break;             // uniform across the CTA
                 uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + c0), r);
+                tmem_ld32(t_row + (uint32_t)c0, r);
                 if (!row_ok) continue;
                 const int col0 = n0 + c0;
-                int32_t v[32];
+                const bool full = col0 + 32 <= p.N;
+                if (CORR) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    int32_t a = p.mul * (int32_t)r[j] + rsa;
-                    if (p.rs_b && col0 + j < p.N) a += p.cb * __ldg(p.rs_b + col0 + j);
-                    v[j] = a;
+                    for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(p.mul * (int32_t)r[j] + rsa + cbt[c0 + j]);
                 }
                 if (p.acc) {
                     int32_t *dst = p.acc + (long long)row * p.N + col0;
-                    if (vec_ok_acc && col0 + 32 <= p.N) {
+                    if (vec_acc && full) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<int4 *>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            *reinterpret_cast<uint4 *>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
                     } else {
-                        for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = v[j];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) dst[j] = (int32_t)r[j];
                     }
                 }
                 if (p.y) {
-                    float f[32];
+                    // y = (sx * sw) * acc, each product rounded to binary32
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float swj = (col0 + j < p.N) ? __ldg(p.sw + col0 + j) : 0.0f;
-                        f[j] = __fmul_rn(__fmul_rn(sxr, swj), (float)v[j]);
-                    }
+                    for (int j = 0; j < 32; ++j)
+                        r[j] = __float_as_uint(__fmul_rn(__fmul_rn(sxr, swt[c0 + j]), (float)(int32_t)r[j]));
                     if (p.y_dtype == QUEST_BF16) {
                         __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.y) + (long long)row * p.ldy + col0;
-                        if (vec_ok_bf16 && col0 + 32 <= p.N) {
+                        if (vec_y && full) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 8) {
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[j], f[j + 1]);
-                                __nv_bfloat162 h1 = __floats2bfloat162_rn(f[j + 2], f[j + 3]);
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[j + 4], f[j + 5]);
-                                __nv_bfloat162 h3 = __floats2bfloat162_rn(f[j + 6], f[j + 7]);
                                 uint4 q;
-                                q.x = *reinterpret_cast<uint32_t *>(&h0);
-                                q.y = *reinterpret_cast<uint32_t *>(&h1);
-                                q.z = *reinterpret_cast<uint32_t *>(&h2);
-                                q.w = *reinterpret_cast<uint32_t *>(&h3);
+                                __nv_bfloat162 h;
+                                h = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+                                q.x = *reinterpret_cast<uint32_t *>(&h);
+                                h = __floats2bfloat162_rn(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                                q.y = *reinterpret_cast<uint32_t *>(&h);
+                                h = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+                                q.z = *reinterpret_cast<uint32_t *>(&h);
+                                h = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+                                q.w = *reinterpret_cast<uint32_t *>(&h);
                                 *reinterpret_cast<uint4 *>(dst + j) = q;
                             }
                         } else {
-                            for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __float2bfloat16_rn(f[j]);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
                         }
                     } else {
                         float *dst = reinterpret_cast<float *>(p.y) + (long long)row * p.ldy + col0;
-                        if (vec_ok_f32 && col0 + 32 <= p.N) {
+                        if (vec_y && full) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4 *>(dst + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
                         } else {
-                            for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = f[j];
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]);
                         }
                     }
                 }
@@ -440,11 +472,11 @@ int make_operand_map(CUtensorMap *tm, const int8_t *base, int64_t rows, int64_t 
     return QUEST_OK;
 }
 
-template <int BN>
+template <int BN, bool CORR>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, CORR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SmemLayout<BN>::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
         attr_done = true;
@@ -454,7 +486,7 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmPar
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
-    gemm_i8_kernel<BN><<<grid, NUM_THREADS, SmemLayout<BN>::TOTAL, st>>>(tmA, tmB, p);
+    gemm_i8_kernel<BN, CORR><<<grid, NUM_THREADS, SmemLayout<BN>::TOTAL, st>>>(tmA, tmB, p);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
@@ -526,7 +558,9 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
     if (s) return s;
     s = make_operand_map(&tmB, b8, N, K, wide ? 256 : 128);
     if (s) return s;
-    return wide ? launch_gemm_bn<256>(tmA, tmB, p, st) : launch_gemm_bn<128>(tmA, tmB, p, st);
+    const bool corr = (bits_x == 8) || (bits_w == 8);
+    if (wide) return corr ? launch_gemm_bn<256, true>(tmA, tmB, p, st) : launch_gemm_bn<256, false>(tmA, tmB, p, st);
+    return corr ? launch_gemm_bn<128, true>(tmA, tmB, p, st) : launch_gemm_bn<128, false>(tmA, tmB, p, st);
 }
 
 }  // namespace quest

@@ -58,6 +58,13 @@ def test_bf16_rows(bits, g, cols):
     check(rows_of("student", 67, cols, bits * 100 + g, True), bits, g)
 
 
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("dtype_bf16", [False, True])
+@pytest.mark.parametrize("g,cols", [(8, 8), (8, 24), (1, 40), (8, 72), (8, 136), (4, 1000), (8, 4104), (2, 16376)])
+def test_row_lengths_that_are_not_multiples_of_32(bits, dtype_bf16, g, cols):
+    check(rows_of("outliers", 19, cols, bits + cols, dtype_bf16), bits, g)
+
+
 @pytest.mark.parametrize("bits", [1, 4, 8])
 @pytest.mark.parametrize("g,cols", [(16, 48), (128, 1280), (512, 512), (2048, 2048), (8192, 8192), (16384, 16384)])
 def test_f32_rows(bits, g, cols):
