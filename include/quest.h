@@ -52,7 +52,8 @@ typedef enum quest_status {
     QUEST_ERR_OVERFLOW = 9,       /* K*(2^bx-1)*(2^bw-1) does not fit in int32 */
     QUEST_ERR_DEVICE = 10,        /* current device is not compute capability 10.x */
     QUEST_ERR_CUDA = 11,          /* a CUDA runtime/driver call failed; see quest_last_cuda_error() */
-    QUEST_ERR_DEVICE_TIMEOUT = 12 /* a bounded wait inside a kernel expired (see quest_device_status) */
+    QUEST_ERR_DEVICE_TIMEOUT = 12,/* a bounded wait inside a kernel expired (see quest_device_status) */
+    QUEST_ERR_STATIC_LIMIT = 13   /* quest_lowbit_gemm_static: problem needs more than QUEST_STATIC_SCRATCH_BYTES */
 } quest_status;
 
 enum { QUEST_F32 = 0, QUEST_BF16 = 1 };
@@ -111,6 +112,34 @@ int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
                       int64_t M, int64_t N, int64_t K,
                       void *y, int y_dtype, int64_t ldy_elems, int32_t *acc,
                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * quest_lowbit_gemm_static -- quest_lowbit_gemm without a workspace argument.  The paper has no
+ * counterpart: this exists for callers that cannot allocate device memory, such as a plug-in that
+ * only receives input and output pointers from its host application, a server that handed all of
+ * device memory to its own pools at start-up (a later cudaMalloc would fail), or a loop that cannot
+ * afford the device-wide synchronisation an allocation implies.  The int8 operands go to a fixed
+ * array of QUEST_STATIC_SCRATCH_BYTES inside the library image; each GPU that loads the library holds
+ * that much memory until the process exits.
+ *
+ *   Arguments, results and error codes are those of quest_lowbit_gemm (caller still passes codes,
+ *   scales and outputs).  In addition QUEST_ERR_STATIC_LIMIT is returned, before anything is
+ *   launched, when quest_workspace_bytes(M, N, K, bits_x, bits_w) exceeds
+ *   QUEST_STATIC_SCRATCH_BYTES, i.e. roughly when (M + N) * K > 4 Mi elements.
+ *   The call itself allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *   The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
+ *   with that device current); make that first call outside any stream capture.
+ *   All calls in the process share the one array per device and it keeps whatever the last call
+ *   left there.  Nothing in it has to start at zero (every byte the kernels read is rewritten by the
+ *   same call first), but two calls whose kernels overlap on the GPU (different streams, or
+ *   different host threads) race on it and produce garbage: serialise them on one stream.
+ */
+#define QUEST_STATIC_SCRATCH_BYTES (4u << 20)
+int quest_lowbit_gemm_static(const uint8_t *xq, const float *sx, int bits_x,
+                             const uint8_t *wq, const float *sw, int bits_w,
+                             int64_t M, int64_t N, int64_t K,
+                             void *y, int y_dtype, int64_t ldy_elems, int32_t *acc,
+                             void *stream);
 
 /*
  * quest_linear_fwd -- Algorithm 1 end to end: quantize x rows, quantize w rows (unless cached),

@@ -135,6 +135,28 @@ def quest_lowbit_gemm(xq: torch.Tensor, sx: torch.Tensor, bits_x: int,
     return y, acc
 
 
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def quest_lowbit_gemm_static(xq: torch.Tensor, sx: torch.Tensor, bits_x: int,
+                             wq: torch.Tensor, sw: torch.Tensor, bits_w: int, K: int,
+                             y: torch.Tensor = None, acc: torch.Tensor = None):
+    """``quest_lowbit_gemm`` for callers that cannot allocate: the int8 operands go to a fixed
+    array inside the library instead of a workspace tensor.  The caller passes every output
+    (``y`` and/or ``acc``) preallocated, so neither this wrapper nor the library allocates.
+    Raises ``QuestError`` (status 13) when (M + N) * K needs more than ``STATIC_SCRATCH_BYTES``.
+    Calls share the one array per device: keep them on one stream."""
+    _require_cuda(xq, sx, wq, sw, y, acc)
+    if y is None and acc is None:
+        raise ValueError("quest_lowbit_gemm_static: pass y and/or acc preallocated")
+    M, N = xq.shape[0], wq.shape[0]
+    st = _lib.load().quest_lowbit_gemm_static(_p(xq), _p(sx), bits_x, _p(wq), _p(sw), bits_w, M, N, K,
+                                              _p(y), _dtype_code(y) if y is not None else 0,
+                                              y.stride(0) if y is not None else N, _p(acc), _stream())
+    _lib.check(st)
+    return y, acc
+
+
 def quest_linear_fwd(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int, trust_factor: float = 1.0,
                      out_dtype=None, y: torch.Tensor = None, saved: dict = None, w_cached: dict = None,
                      workspace: torch.Tensor = None, want_masks: bool = True) -> dict:

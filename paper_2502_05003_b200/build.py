@@ -21,6 +21,7 @@ UNITS = {
     "quest_api.cu": [],
     "quest_quantize.cu": ["-fmad=false"],
     "quest_gemm.cu": [],
+    "quest_static.cu": [],
 }
 
 

@@ -142,6 +142,7 @@ const char *quest_status_string(int status) {
         case QUEST_ERR_DEVICE: return "current device is not compute capability 10.x";
         case QUEST_ERR_CUDA: return "CUDA call failed";
         case QUEST_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case QUEST_ERR_STATIC_LIMIT: return "problem too large for the library's static scratch (QUEST_STATIC_SCRATCH_BYTES)";
         default: return "unknown status";
     }
 }
