@@ -98,7 +98,7 @@ int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64
  *
  *   xq, sx, bits_x   device: codes [M x K] and scales [M] of the activations
  *   wq, sw, bits_w   device: codes [N x K] and scales [N] of the weights (both operands K-major)
- *   M, N, K          M, N >= 0; K >= 32, K % 32 == 0; K*(2^bx-1)*(2^bw-1) < 2^31
+ *   M, N, K          M, N >= 0; 32 <= K <= 65504, K % 32 == 0; K*(2^bx-1)*(2^bw-1) < 2^31
  *   y, y_dtype, ldy  device out [M x N], row stride ldy elements, QUEST_F32 or QUEST_BF16;
  *                    may be NULL if only acc is wanted
  *   acc              device out, dense [M x N] int32 raw accumulators; may be NULL

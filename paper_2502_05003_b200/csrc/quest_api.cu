@@ -101,7 +101,7 @@ static int validate_quantize(const void *x, int dtype, int64_t rows, int64_t col
 static int validate_gemm_shape(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w) {
     if (bits_x < 1 || bits_x > 8 || bits_w < 1 || bits_w > 8) return QUEST_ERR_BITS;
     if (M < 0 || N < 0 || M > (int64_t)1 << 30 || N > (int64_t)1 << 30 || K < 32 || K % 32 != 0 ||
-        K > (int64_t)1 << 24)
+        K > 65504)
         return QUEST_ERR_SHAPE;
     const int64_t worst = K * (((int64_t)1 << bits_x) - 1) * (((int64_t)1 << bits_w) - 1);
     if (worst >= ((int64_t)1 << 31)) return QUEST_ERR_OVERFLOW;
@@ -206,9 +206,10 @@ int quest_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t
     int s = validate_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, codes, mask);
     if (s) return s;
     if ((s = check_device())) return s;
+    if (rows == 0) return QUEST_OK;
     StageScope scope(QUEST_STAGE_QUANT_X, reinterpret_cast<cudaStream_t>(stream));
-    return launch_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, codes, scales, mask,
-                           nullptr, reinterpret_cast<cudaStream_t>(stream));
+    const QuantJob job = {x, rows, ld_elems, codes, scales, mask, nullptr, nullptr};
+    return launch_quantize(&job, 1, dtype, cols, bits, had_block, trust_factor, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
@@ -217,8 +218,9 @@ int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64
     int s = validate_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, nullptr, mask);
     if (s) return s;
     if ((s = check_device())) return s;
-    return launch_quantize(x, dtype, rows, cols, ld_elems, bits, had_block, trust_factor, nullptr, nullptr, mask,
-                           nullptr, reinterpret_cast<cudaStream_t>(stream));
+    if (rows == 0) return QUEST_OK;
+    const QuantJob job = {x, rows, ld_elems, nullptr, nullptr, mask, nullptr, nullptr};
+    return launch_quantize(&job, 1, dtype, cols, bits, had_block, trust_factor, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
@@ -275,21 +277,20 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     Workspace ws = carve_workspace(workspace, M, N, K);
     const bool need_rs = bits == 8;
-    // activations: codes, scale, mask and the int8 operand in one pass
-    {
-        StageScope scope(QUEST_STAGE_QUANT_X, st);
-        if ((s = launch_quantize(x, dtype, M, K, K, bits, had_block, trust_factor, xq, sx, mx, ws.a8, st))) return s;
-    }
+    // codes, scale, mask, the int8 operand (and its row sums for 8-bit codes) in one pass; x and w
+    // share one launch when both are quantized
+    const QuantJob jx = {x, M, K, xq, sx, mx, ws.a8, need_rs ? ws.rs_a : nullptr};
     if (w_is_cached) {
+        {
+            StageScope scope(QUEST_STAGE_QUANT_X, st);
+            if ((s = launch_quantize(&jx, 1, dtype, K, bits, had_block, trust_factor, st))) return s;
+        }
         StageScope scope(QUEST_STAGE_UNPACK, st);
         if ((s = launch_unpack(wq, bits, N, K, ws.b8, need_rs ? ws.rs_b : nullptr, st))) return s;
     } else {
-        StageScope scope(QUEST_STAGE_QUANT_W, st);
-        if ((s = launch_quantize(w, dtype, N, K, K, bits, had_block, trust_factor, wq, sw, mw, ws.b8, st))) return s;
-    }
-    if (need_rs) {
-        if ((s = launch_rowsum(ws.a8, M, K, ws.rs_a, st))) return s;
-        if (!w_is_cached && (s = launch_rowsum(ws.b8, N, K, ws.rs_b, st))) return s;
+        StageScope scope(QUEST_STAGE_QUANT_X, st);
+        const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, ws.b8, need_rs ? ws.rs_b : nullptr}};
+        if ((s = launch_quantize(jobs, 2, dtype, K, bits, had_block, trust_factor, st))) return s;
     }
     StageScope scope(QUEST_STAGE_GEMM, st);
     return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits, bits, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);

@@ -5,7 +5,8 @@
 //
 // B200 has no dense 4-bit integer MMA, so the contraction runs as tcgen05.mma kind::i8 on int8
 // operand values held in a caller-provided workspace (written either by the quantizer itself or
-// by unpack_codes_kernel below).  For b < 8 the operand value is the grid value c = 2k-(2^b-1);
+// by unpack_codes_kernel below).  For b < 8 the operand value is 2^(7-b) times the grid value
+// c = 2k-(2^b-1) (quest_operand.cuh) and the epilogue shifts the exact power of two back out;
 // for b = 8 (|c| up to 255) it is v = k - 128 and the epilogue restores
 // c_x . c_w = 4 v_x.v_w + 2 sum(v_x) + 2 sum(v_w) + K exactly from per-row sums.
 //
@@ -23,6 +24,7 @@
 #include <cuda_bf16.h>
 
 #include "quest_internal.cuh"
+#include "quest_operand.cuh"
 
 namespace quest {
 namespace {
@@ -42,8 +44,8 @@ struct GemmParams {
     const float *sw;
     const int32_t *rs_a;   // row sums of the A operand values (nullable)
     const int32_t *rs_b;   // row sums of the B operand values (nullable)
-    int mul;               // acc' = mul*acc + ca*rs_a[i] + cb*rs_b[j] + ck
-    int ca, cb, ck;
+    int mul;               // acc' = (mul*acc + ca*rs_a[i] + cb*rs_b[j] + ck) >> sh   (exact)
+    int ca, cb, ck, sh;
     void *y;
     int y_dtype;
     long long ldy;
@@ -323,7 +325,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const bool full = col0 + 32 <= p.N;
                 if (CORR) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = (uint32_t)(p.mul * (int32_t)r[j] + rsa + cbt[c0 + j]);
+                    for (int j = 0; j < 32; ++j)
+                        r[j] = (uint32_t)((int32_t)((uint32_t)p.mul * r[j] + (uint32_t)rsa + (uint32_t)cbt[c0 + j]) >> p.sh);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = (uint32_t)((int32_t)r[j] >> p.sh);
                 }
                 if (p.acc) {
                     int32_t *dst = p.acc + (long long)row * p.N + col0;
@@ -393,33 +399,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Packed codes -> int8 operand values (and row sums for 8-bit codes).
-// One thread converts 32 consecutive elements (rows are dense and K % 32 == 0).
+// Packed codes -> int8 operand values (quest_operand.cuh).  One thread converts 32 consecutive
+// elements (rows are dense and K % 32 == 0).
 // ---------------------------------------------------------------------------------------------
+template <int CB>
 __global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits, long long n_groups,
                                     int8_t *__restrict__ out) {
-    const int cb = container_bits(bits);
-    const int L1 = (1 << bits) - 1;
-    const int words = cb;                                   // 32 elements * cb bits = cb 32-bit words
     for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n_groups;
          g += (long long)gridDim.x * blockDim.x) {
-        const uint32_t *src = reinterpret_cast<const uint32_t *>(codes) + g * words;
-        uint32_t w[8];
-        for (int i = 0; i < words; ++i) w[i] = __ldg(src + i);
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(codes) + g * CB;
+        uint32_t w[CB];
+#pragma unroll
+        for (int i = 0; i < CB; ++i) w[i] = __ldg(src + i);
         uint32_t o[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            uint32_t packed = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int e = q * 4 + j;
-                const int bitpos = e * cb;
-                const int k = (w[bitpos >> 5] >> (bitpos & 31)) & ((1 << cb) - 1);
-                const int v = (bits == 8) ? (k - 128) : (2 * k - L1);
-                packed |= (uint32_t)(uint8_t)(int8_t)v << (8 * j);
-            }
-            o[q] = packed;
-        }
+        operand_from_code_words<CB>(w, bits, o);
         uint4 *dst = reinterpret_cast<uint4 *>(out + g * 32);
         dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
         dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -517,7 +510,12 @@ int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_
     const int threads = 256;
     long long blocks = (n_groups + threads - 1) / threads;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    unpack_codes_kernel<<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out);
+    switch (container_bits(bits)) {
+        case 1: unpack_codes_kernel<1><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
+        case 2: unpack_codes_kernel<2><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
+        case 4: unpack_codes_kernel<4><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
+        default: unpack_codes_kernel<8><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e);
     if (rowsum) return launch_rowsum(out, rows, K, rowsum, st);
@@ -537,18 +535,17 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
                 int32_t *acc, cudaStream_t st) {
     if (M == 0 || N == 0) return QUEST_OK;
-    // operand value v relates to the grid value c by c = m*v + a: (1, 0) below 8 bits, (2, 1) at 8 bits
-    const int mx = bits_x == 8 ? 2 : 1, ax = bits_x == 8 ? 1 : 0;
-    const int mw = bits_w == 8 ? 2 : 1, aw = bits_w == 8 ? 1 : 0;
+    // operand value v relates to the grid value c by v = 2^(7-b) c below 8 bits and c = 2v + 1 at 8 bits
+    const bool x8 = bits_x == 8, w8 = bits_w == 8;
     GemmParams p;
     p.M = (int)M; p.N = (int)N; p.K = (int)K;
     p.sx = sx; p.sw = sw;
-    p.mul = mx * mw;
-    p.ca = mx * aw;                        // multiplies sum_k v_x[i][k]
-    p.cb = ax * mw;                        // multiplies sum_k v_w[j][k]
-    p.ck = ax * aw * (int)K;
-    p.rs_a = p.ca ? rs_a : nullptr;
-    p.rs_b = p.cb ? rs_b : nullptr;
+    if (!x8 && !w8) { p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 14 - bits_x - bits_w; }
+    else if (x8 && w8) { p.mul = 4; p.ca = 2; p.cb = 2; p.ck = (int)K; p.sh = 0; }
+    else if (x8) { p.mul = 2; p.ca = 0; p.cb = 1; p.ck = 0; p.sh = 7 - bits_w; }   // 2 sum v_x op_w + sum op_w
+    else { p.mul = 2; p.ca = 1; p.cb = 0; p.ck = 0; p.sh = 7 - bits_x; }
+    p.rs_a = p.ca ? rs_a : nullptr;                      // row sums of the x operand bytes
+    p.rs_b = p.cb ? rs_b : nullptr;                      // row sums of the w operand bytes
     p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;

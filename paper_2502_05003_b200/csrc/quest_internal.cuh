@@ -57,9 +57,21 @@ int *device_status_word();                // device address of the timeout word 
 int check_device();                       // QUEST_OK iff current device is sm_10x
 
 // Launchers (each returns a quest_status; arguments already validated).
-int launch_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
-                    int bits, int had_block, float trust_factor,
-                    uint8_t *codes, float *scales, uint8_t *mask, int8_t *op8, cudaStream_t st);
+// One tensor of a quantizer launch: rows of `x` -> any of codes / scales / mask / int8 GEMM
+// operand / per-row sum of the operand bytes (each nullable).
+struct QuantJob {
+    const void *x;
+    int64_t rows;
+    int64_t ld;
+    uint8_t *codes;
+    float *scales;
+    uint8_t *mask;
+    int8_t *op8;
+    int32_t *rowsum;
+};
+// Up to two tensors with the same row length, dtype and parameters share one launch.
+int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
+                    float trust_factor, cudaStream_t st);
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out,
                   int32_t *rowsum, cudaStream_t st);
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st);

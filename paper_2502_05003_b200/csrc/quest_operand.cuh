@@ -1,0 +1,92 @@
+// int8 tensor-core operand values from packed level indices (device code shared by the quantizer
+// and the unpack kernel of the low-bit GEMM).
+//
+// For b < 8 the operand byte of level k is the top-aligned offset-binary code with half an LSB
+// set,  v = ((k << (8-b)) | (1 << (7-b))) ^ 0x80  =  2^(7-b) * c   with c = 2k - (2^b - 1)
+// the grid value of Eq. 1: an exact power-of-two multiple of c that fits int8 (|v| <= 127) and
+// costs one shift and one three-input logic operation per four elements.  The contraction of two
+// such operands is 2^(14-bx-bw) * sum_k cx cw; the GEMM epilogue shifts it back (exact).
+// For b = 8 (|c| up to 255) the operand is v = k - 128 = k ^ 0x80 and the epilogue restores the
+// grid-value product from per-row sums of v.
+#pragma once
+#include <stdint.h>
+
+namespace quest {
+
+__host__ __device__ inline int operand_shift(int bits) { return bits == 8 ? 0 : 7 - bits; }
+
+__device__ __forceinline__ uint32_t lop3_mask_xor_set(uint32_t x, uint32_t m, uint32_t c) {
+    // per bit: m ? x ^ c : c
+    return ((x ^ c) & m) | (c & ~m);
+}
+__device__ __forceinline__ uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel) { return __byte_perm(a, b, sel); }
+
+// 4x4 byte transpose: in[j] holds bytes (e_j, e_{4+j}, e_{8+j}, e_{12+j}); out[m] = (e_{4m}, .., e_{4m+3}).
+__device__ __forceinline__ void transpose4x4(const uint32_t (&in)[4], uint32_t (&out)[4]) {
+    const uint32_t a = byte_perm(in[0], in[1], 0x5140);   // (e0, e1, e4, e5)
+    const uint32_t b = byte_perm(in[2], in[3], 0x5140);   // (e2, e3, e6, e7)
+    const uint32_t c = byte_perm(in[0], in[1], 0x7362);   // (e8, e9, e12, e13)
+    const uint32_t d = byte_perm(in[2], in[3], 0x7362);   // (e10, e11, e14, e15)
+    out[0] = byte_perm(a, b, 0x5410);
+    out[1] = byte_perm(a, b, 0x7632);
+    out[2] = byte_perm(c, d, 0x5410);
+    out[3] = byte_perm(c, d, 0x7632);
+}
+
+// 32 consecutive codes (CB words of CB-bit containers, element 0 lowest) -> 32 operand bytes in
+// element order (8 words).
+template <int CB>
+__device__ __forceinline__ void operand_from_code_words(const uint32_t (&w)[CB], int bits, uint32_t (&o)[8]) {
+    if constexpr (CB == 8) {
+        if (bits == 8) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) o[q] = w[q] ^ 0x80808080u;
+        } else {
+            const uint32_t m = (0xFFu << (8 - bits)) & 0xFFu;
+            const uint32_t M = m * 0x01010101u, C = (0x80u | (1u << (7 - bits))) * 0x01010101u;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) o[q] = lop3_mask_xor_set(w[q] << (8 - bits), M, C);
+        }
+    } else if constexpr (CB == 4) {
+        const int up = 4 - bits;                               // 0 at b = 4, 1 at b = 3
+        const uint32_t m = (0xFFu << (8 - bits)) & 0xFFu;
+        const uint32_t M = m * 0x01010101u, C = (0x80u | (1u << (7 - bits))) * 0x01010101u;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t lo = lop3_mask_xor_set(w[q] << (4 + up), M, C);   // elements 0, 2, 4, 6 of the word
+            const uint32_t hi = lop3_mask_xor_set(w[q] << up, M, C);         // elements 1, 3, 5, 7
+            o[2 * q] = byte_perm(lo, hi, 0x5140);
+            o[2 * q + 1] = byte_perm(lo, hi, 0x7362);
+        }
+    } else if constexpr (CB == 2) {
+        const uint32_t M = 0xC0C0C0C0u, C = 0xA0A0A0A0u;       // b = 2: (k << 6 | 32) ^ 128
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            uint32_t x[4], t[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[j] = lop3_mask_xor_set(w[q] << (6 - 2 * j), M, C);
+            transpose4x4(x, t);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) o[4 * q + j] = t[j];
+        }
+    } else {
+        const uint32_t M = 0x80808080u, C = 0xC0C0C0C0u;       // b = 1: (k << 7 | 64) ^ 128
+        uint32_t x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = lop3_mask_xor_set(w[0] << (7 - j), M, C);   // bytes (e_j, e_{8+j}, e_{16+j}, e_{24+j})
+        // two 4x4 transposes give, for m = 0..3, elements 8m..8m+3 and 8m+4..8m+7
+        uint32_t a[4] = {x[0], x[1], x[2], x[3]}, b[4] = {x[4], x[5], x[6], x[7]}, ta[4], tb[4];
+        transpose4x4(a, ta);
+        transpose4x4(b, tb);
+#pragma unroll
+        for (int m2 = 0; m2 < 4; ++m2) {
+            o[2 * m2] = ta[m2];
+            o[2 * m2 + 1] = tb[m2];
+        }
+    }
+}
+
+// Sum of the four signed bytes of a word.
+__device__ __forceinline__ int sum_bytes_s8(uint32_t w) { return __dp4a((int)w, 0x01010101, 0); }
+
+}  // namespace quest

@@ -9,6 +9,7 @@
 // trusted = |t - level| <= trust_factor/2.  This file is compiled with -fmad=false and uses
 // the explicit _rn intrinsics so that the compiler cannot fuse or reorder any of it.
 #include "quest_internal.cuh"
+#include "quest_operand.cuh"
 
 namespace quest {
 
@@ -98,7 +99,7 @@ quantize_generic_kernel(const void *__restrict__ x, int dtype, int64_t rows, int
                 const int k = round_level(u[grp * 8 + j], inv, qc, trusted);
                 packed |= (uint64_t)k << (j * cb);
                 mbits |= (trusted ? 1u : 0u) << j;
-                v8[j] = (int8_t)(bits == 8 ? k - 128 : 2 * k - L1);
+                v8[j] = (int8_t)(bits == 8 ? k - 128 : (2 * k - L1) << (7 - bits));   // see quest_operand.cuh
             }
             if (codes) {
                 uint8_t *cr = codes + row * (int64_t)(cols * cb / 8) + (int64_t)grp * cb;
@@ -117,141 +118,152 @@ quantize_generic_kernel(const void *__restrict__ x, int dtype, int64_t rows, int
 
 
 // ---------------------------------------------------------------------------------------------
-// Row kernel: every thread owns 32 CONTIGUOUS elements of a row (cols % 32 == 0).
-//   * butterflies of stride >= 1024 go through shared memory (rows wider than a warp's span),
-//     strides 32..512 through warp shuffles, strides 16..1 stay in registers -- descending
+// Row kernel: every thread owns E CONTIGUOUS elements of a row (E = 64 or 32, cols % E == 0),
+// held as E/2 float2 pairs so that most of the arithmetic runs on the packed binary32 pipe
+// (two IEEE operations per instruction, each rounded exactly like the scalar form).
+//   * butterflies whose partner is in another warp (stride >= 32 E) go through shared memory,
+//     strides E .. 16 E through warp shuffles, strides E/2 .. 1 stay in registers -- descending
 //     stride overall, which is the canonical order;
 //   * the sum of squares is reduced pairwise in the thread, then over lanes, then over warps;
-//   * rounding, the trust test and the packing work on the thread's 32 elements, so each
-//     thread stores whole words: 32*container/8 bytes of codes, 4 bytes of mask, 32 operand bytes.
-// A row of T = cols/32 threads occupies S slots of the CTA: the next power of two if T < 32,
-// else T rounded up to whole warps; slots past T carry zeros, which is the zero padding of the
-// canonical pairwise sum.
+//   * rounding, the trust test and the packing work on groups of 32 elements, so each thread
+//     stores whole words: 4 bytes of mask, 32*container/8 bytes of codes, 32 operand bytes;
+//   * the int8 GEMM operand is derived from the packed code words (quest_operand.cuh).
+// A row of T = cols/E threads occupies S slots of the CTA: the next power of two if T < 32, else
+// T rounded up to whole warps; slots past T carry zeros, which is the zero padding of the
+// canonical pairwise sum.  One launch can serve two tensors of the same row length (x and w of a
+// linear layer): the first `blocks0` CTAs work on tensor 0, the rest on tensor 1.
 // ---------------------------------------------------------------------------------------------
 #define QUEST_MAGIC_RNE 12582912.0f            /* 1.5 * 2^23: x + MAGIC rounds x to an integer (ties to even) */
 #define QUEST_MAGIC_BITS 0x4B400000u
 
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-// (a, b) -> (a + b, a - b) on two independent lanes with the packed binary32 instructions
-__device__ __forceinline__ void butterfly2(float &a0, float &a1, float &b0, float &b1) {
-    const uint64_t A = pack2(a0, a1), B = pack2(b0, b1);
-    uint64_t S, D;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(S) : "l"(A), "l"(B));
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(D) : "l"(A), "l"(B));
-    unpack2(S, a0, a1);
-    unpack2(D, b0, b1);
-}
-// own * sgn + partner on two lanes (sgn = +-1: an exact add or subtract, one rounding)
-__device__ __forceinline__ void fma2(float &x0, float &x1, float s, float p0, float p1) {
-    const uint64_t X = pack2(x0, x1), Sg = pack2(s, s), P = pack2(p0, p1);
-    uint64_t R;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(R) : "l"(X), "l"(Sg), "l"(P));
-    unpack2(R, x0, x1);
-}
+struct QuantTensor {
+    const void *x;
+    long long rows;
+    long long ld;
+    uint8_t *codes;
+    float *scales;
+    uint8_t *mask;
+    int8_t *op8;
+    int32_t *rowsum;       // sum of the row's operand bytes (needed by the GEMM for 8-bit codes)
+};
+struct QuantArgs {
+    QuantTensor t[2];
+    int blocks0;
+    int cols, bits, had_block;
+    QuantConsts qc;
+    int S, R;
+};
 
-template <bool BF16, int CB>
-__global__ void __launch_bounds__(512)
-quantize_row32_kernel(const void *__restrict__ x, int64_t rows, int cols, int64_t ld, int bits, int had_block,
-                      QuantConsts qc, int S, int R,
-                      uint8_t *__restrict__ codes, float *__restrict__ scales, uint8_t *__restrict__ mask,
-                      int8_t *__restrict__ op8) {
-    extern __shared__ float xsm[];                 // [32][blockDim.x] exchange, then [warps] partial sums
+template <bool BF16, int CB, int E>
+__global__ void __launch_bounds__(E == 64 ? 256 : 512)
+quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
+    extern __shared__ float xsm[];                 // [E][blockDim.x] exchange, then [warps] partial sums
+    constexpr int H = E / 2;                       // float2 pairs per thread
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int nthreads = blockDim.x;
+    const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
+    const QuantTensor &tn = a.t[which];
+    const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
+    const int S = a.S;
     const int r_local = tid / S;
     const int tr = tid - r_local * S;              // slot inside the row
-    const int64_t row = (int64_t)blockIdx.x * R + r_local;
-    const int T = cols >> 5;
-    const bool active = (row < rows) && (tr < T);
+    const long long row = (long long)blk * a.R + r_local;
+    const int cols = a.cols;
+    const int had_block = a.had_block;
+    const int T = cols / E;
+    const bool active = (row < tn.rows) && (tr < T);
 
-    float v[32];
+    float2 v[H];
     if (active) {
         if (BF16) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(x) + row * ld + tr * 32);
+            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(tn.x) + row * tn.ld + (long long)tr * E);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < E / 8; ++q) {
                 const uint4 w = __ldg(src + q);
                 const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    v[q * 8 + 2 * j] = __uint_as_float(ww[j] << 16);
-                    v[q * 8 + 2 * j + 1] = __uint_as_float(ww[j] & 0xFFFF0000u);
-                }
+                for (int j = 0; j < 4; ++j)
+                    v[q * 4 + j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
             }
         } else {
-            const float4 *src = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(x) + row * ld + tr * 32);
+            const float4 *src = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(tn.x) + row * tn.ld + (long long)tr * E);
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
+            for (int q = 0; q < E / 4; ++q) {
                 const float4 w = __ldg(src + q);
-                v[q * 4] = w.x; v[q * 4 + 1] = w.y; v[q * 4 + 2] = w.z; v[q * 4 + 3] = w.w;
+                v[q * 2] = make_float2(w.x, w.y);
+                v[q * 2 + 1] = make_float2(w.z, w.w);
             }
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = 0.0f;
+        for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
     }
 
     // ---- rotation, descending stride --------------------------------------------------------
-    for (int s = had_block >> 1; s >= 1024; s >>= 1) {        // partner thread is in another warp
-        const int dist = s >> 5;
+    const float2 neg1 = make_float2(-1.0f, -1.0f);
+    for (int s = had_block >> 1; s >= 32 * E; s >>= 1) {      // partner thread is in another warp
+        const int dist = s / E;
+        float2 *x2 = reinterpret_cast<float2 *>(xsm);
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) xsm[i * nthreads + tid] = v[i];
+        for (int i = 0; i < H; ++i) x2[i * nthreads + tid] = v[i];
         __syncthreads();
-        const float sgn = (tid & dist) ? -1.0f : 1.0f;
+        const float sg = (tid & dist) ? -1.0f : 1.0f;
+        const float2 sgn = make_float2(sg, sg);
         const int pt = tid ^ dist;
 #pragma unroll
-        for (int i = 0; i < 32; i += 2)
-            fma2(v[i], v[i + 1], sgn, xsm[i * nthreads + pt], xsm[(i + 1) * nthreads + pt]);
+        for (int i = 0; i < H; ++i) v[i] = __ffma2_rn(v[i], sgn, x2[i * nthreads + pt]);
     }
     {
         int s0 = had_block >> 1;
-        if (s0 > 512) s0 = 512;
+        if (s0 > 16 * E) s0 = 16 * E;
 #pragma unroll 1
-        for (int s = s0; s >= 32; s >>= 1) {                   // partner thread is a lane of this warp
-            const int dist = s >> 5;
-            const float sgn = (lane & dist) ? -1.0f : 1.0f;
+        for (int s = s0; s >= E; s >>= 1) {                    // partner thread is a lane of this warp
+            const int dist = s / E;
+            const float sg = (lane & dist) ? -1.0f : 1.0f;
+            const float2 sgn = make_float2(sg, sg);
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-                const float p0 = __shfl_xor_sync(0xffffffffu, v[i], dist);
-                const float p1 = __shfl_xor_sync(0xffffffffu, v[i + 1], dist);
-                fma2(v[i], v[i + 1], sgn, p0, p1);
+            for (int i = 0; i < H; ++i) {
+                float2 p;
+                p.x = __shfl_xor_sync(0xffffffffu, v[i].x, dist);
+                p.y = __shfl_xor_sync(0xffffffffu, v[i].y, dist);
+                v[i] = __ffma2_rn(v[i], sgn, p);               // own * (+-1) + partner: one rounding
             }
         }
     }
 #pragma unroll
-    for (int s = 16; s >= 2; s >>= 1) {                        // partner element is in this thread
+    for (int s = E / 2; s >= 2; s >>= 1) {                     // partner element is in this thread
         if (s < had_block) {
+            const int s2 = s >> 1;
 #pragma unroll
-            for (int i = 0; i < 32; i += 2)
-                if ((i & s) == 0) butterfly2(v[i], v[i + 1], v[i + s], v[i + s + 1]);
+            for (int i = 0; i < H; ++i)
+                if ((i & s2) == 0) {
+                    const float2 p = v[i], q = v[i + s2];
+                    v[i] = __fadd2_rn(p, q);
+                    v[i + s2] = __ffma2_rn(q, neg1, p);        // p - q
+                }
         }
     }
     if (had_block > 1) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-            const float a = v[i], b = v[i + 1];
-            v[i] = __fadd_rn(a, b);
-            v[i + 1] = __fsub_rn(a, b);
+        for (int i = 0; i < H; ++i) {
+            const float p = v[i].x, q = v[i].y;
+            v[i] = make_float2(__fadd_rn(p, q), __fsub_rn(p, q));
         }
     }
 
     // ---- sum of squares: pairwise over adjacent elements, zero-padded row --------------------
     float ss;
     {
-        float q[16];
+        float q[H];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) q[i] = __fadd_rn(__fmul_rn(v[2 * i], v[2 * i]), __fmul_rn(v[2 * i + 1], v[2 * i + 1]));
+        for (int i = 0; i < H; ++i) {
+            const float2 sq = __fmul2_rn(v[i], v[i]);
+            q[i] = __fadd_rn(sq.x, sq.y);
+        }
 #pragma unroll
-        for (int n = 8; n >= 1; n >>= 1)
+        for (int n = H / 2; n >= 1; n >>= 1)
 #pragma unroll
             for (int i = 0; i < n; ++i) q[i] = __fadd_rn(q[2 * i], q[2 * i + 1]);
         ss = q[0];
@@ -271,88 +283,107 @@ quantize_row32_kernel(const void *__restrict__ x, int64_t rows, int cols, int64_
         for (int m = 1; m < nwp2; m <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, m));
     }
     const float rms = __fsqrt_rn(__fdiv_rn(ss, (float)cols));
-    const float inv = (rms > 0.0f) ? __fdiv_rn(qc.A, rms) : 0.0f;
-    if (!active) return;
-    if (scales && tr == 0) scales[row] = __fmul_rn(rms, qc.B);
+    const float inv = (rms > 0.0f) ? __fdiv_rn(a.qc.A, rms) : 0.0f;
+    if (!active && tn.rowsum == nullptr) return;
+    if (active && tn.scales && tr == 0) tn.scales[row] = __fmul_rn(rms, a.qc.B);
 
     // ---- project: level axis, clamp, round to nearest even, trust test -----------------------
-    uint32_t kb[32];                                            // MAGIC_BITS + level
-    uint32_t mbits = 0;
+    const float2 inv2 = make_float2(inv, inv), c02 = make_float2(a.qc.c0, a.qc.c0);
+    const float2 magic2 = make_float2(QUEST_MAGIC_RNE, QUEST_MAGIC_RNE);
+    const float2 nmagic2 = make_float2(-QUEST_MAGIC_RNE, -QUEST_MAGIC_RNE);
+    const float top = a.qc.top, hh = a.qc.h;
+    int rsum = 0;
+    if (active) {
 #pragma unroll
-    for (int i = 31; i >= 0; --i) {
-        const float t = __fmaf_rn(v[i], inv, qc.c0);
-        const float tc = fminf(fmaxf(t, 0.0f), qc.top);
-        const float km = __fadd_rn(tc, QUEST_MAGIC_RNE);
-        const float kf = __fsub_rn(km, QUEST_MAGIC_RNE);
-        const float dlt = __fsub_rn(qc.h, fabsf(__fsub_rn(t, kf)));   // >= +0  <=>  trusted
-        mbits = __funnelshift_l(__float_as_uint(dlt), mbits, 1);         // sign bit: 1 = masked
-        kb[i] = __float_as_uint(km);
-    }
-    mbits = ~mbits;
-    if (mask) reinterpret_cast<uint32_t *>(mask + row * (int64_t)(cols >> 3))[tr] = mbits;
-
-    if (codes) {
-        // pack 32/CB codes per word: sum_j (MAGIC_BITS + k_j) * 2^(CB*j), minus the constant part
-        constexpr int PER = 32 / CB;
-        constexpr int WORDS = CB;
-        uint32_t magic_sum = 0;
+        for (int g32 = 0; g32 < E / 32; ++g32) {
+            uint32_t kb[32];                                    // MAGIC_BITS + level
+            uint32_t mbits = 0;
 #pragma unroll
-        for (int j = 0; j < PER; ++j) magic_sum += QUEST_MAGIC_BITS << (CB * j);
-        uint32_t w[WORDS];
-#pragma unroll
-        for (int q = 0; q < WORDS; ++q) {
-            uint32_t acc = 0;
-#pragma unroll
-            for (int j = PER - 1; j >= 0; --j) acc = (acc << CB) + kb[q * PER + j];
-            w[q] = acc - magic_sum;
-        }
-        uint8_t *dst = codes + row * (int64_t)(cols * CB / 8) + (int64_t)tr * (4 * CB);
-        if constexpr (CB == 8) {
-            reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            reinterpret_cast<uint4 *>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-        } else if constexpr (CB == 4) {
-            reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        } else if constexpr (CB == 2) {
-            reinterpret_cast<uint2 *>(dst)[0] = make_uint2(w[0], w[1]);
-        } else {
-            reinterpret_cast<uint32_t *>(dst)[0] = w[0];
-        }
-    }
-    if (op8) {
-        // int8 operand of the tensor-core contraction: c = 2k - (2^b - 1), or k - 128 at b = 8
-        const int L1 = (1 << bits) - 1;
-        uint32_t o[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            uint32_t acc = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int k = (int)(kb[q * 4 + j] - QUEST_MAGIC_BITS);
-                const int val = (bits == 8) ? (k - 128) : (2 * k - L1);
-                acc |= (uint32_t)(val & 0xFF) << (8 * j);
+            for (int i = 15; i >= 0; --i) {
+                const float2 t = __ffma2_rn(v[g32 * 16 + i], inv2, c02);
+                float2 tc;
+                tc.x = fminf(fmaxf(t.x, 0.0f), top);
+                tc.y = fminf(fmaxf(t.y, 0.0f), top);
+                const float2 km = __fadd2_rn(tc, magic2);
+                const float2 kf = __fadd2_rn(km, nmagic2);
+                const float2 d = __ffma2_rn(kf, neg1, t);                      // t - kf
+                const float dy = __fsub_rn(hh, fabsf(d.y));                    // >= +0  <=>  trusted
+                const float dx = __fsub_rn(hh, fabsf(d.x));
+                mbits = __funnelshift_l(__float_as_uint(dy), mbits, 1);         // sign bit: 1 = masked
+                mbits = __funnelshift_l(__float_as_uint(dx), mbits, 1);
+                kb[2 * i] = __float_as_uint(km.x);
+                kb[2 * i + 1] = __float_as_uint(km.y);
             }
-            o[q] = acc;
+            mbits = ~mbits;
+            if (tn.mask)
+                reinterpret_cast<uint32_t *>(tn.mask + row * (long long)(cols >> 3))[tr * (E / 32) + g32] = mbits;
+
+            // pack 32/CB codes per word: sum_j (MAGIC_BITS + k_j) * 2^(CB*j), minus the constant part
+            constexpr int PER = 32 / CB;
+            uint32_t magic_sum = 0;
+#pragma unroll
+            for (int j = 0; j < PER; ++j) magic_sum += QUEST_MAGIC_BITS << (CB * j);
+            uint32_t w[CB];
+#pragma unroll
+            for (int q = 0; q < CB; ++q) {
+                uint32_t acc = 0;
+#pragma unroll
+                for (int j = PER - 1; j >= 0; --j) acc = (acc << CB) + kb[q * PER + j];
+                w[q] = acc - magic_sum;
+            }
+            if (tn.codes) {
+                uint8_t *dst = tn.codes + row * (long long)(cols * CB / 8) + ((long long)tr * (E / 32) + g32) * (4 * CB);
+                if constexpr (CB == 8) {
+                    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    reinterpret_cast<uint4 *>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                } else if constexpr (CB == 4) {
+                    reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                } else if constexpr (CB == 2) {
+                    reinterpret_cast<uint2 *>(dst)[0] = make_uint2(w[0], w[1]);
+                } else {
+                    reinterpret_cast<uint32_t *>(dst)[0] = w[0];
+                }
+            }
+            if (tn.op8) {
+                uint32_t o[8];
+                operand_from_code_words<CB>(w, a.bits, o);
+                uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                if (tn.rowsum) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) rsum += sum_bytes_s8(o[q]);
+                }
+            }
         }
-        uint4 *dst = reinterpret_cast<uint4 *>(op8 + row * (int64_t)cols + (int64_t)tr * 32);
-        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+    if (tn.rowsum) {                                            // uniform over the CTA
+        for (int m = 1; m < lanes_per_row; m <<= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, m);
+        if (S > 32) {
+            int *ism = reinterpret_cast<int *>(xsm);
+            __syncthreads();
+            if (lane == 0) ism[tid >> 5] = rsum;
+            __syncthreads();
+            if (tr == 0) {
+                rsum = 0;
+                const int w0 = (r_local * S) >> 5;
+                for (int i = 0; i < (S >> 5); ++i) rsum += ism[w0 + i];
+            }
+        }
+        if (active && tr == 0) tn.rowsum[row] = rsum;
     }
 }
 
-template <bool BF16>
-static cudaError_t launch_row32(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st,
-                                const void *x, int64_t rows, int cols, int64_t ld, int bits, int had_block,
-                                QuantConsts qc, int S, int R, uint8_t *codes, float *scales, uint8_t *mask,
-                                int8_t *op8) {
+template <bool BF16, int E>
+static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
         if (smem > 48 * 1024) {                                                                             \
-            cudaError_t e_ = cudaFuncSetAttribute(quantize_row32_kernel<BF16, CBV>,                         \
+            cudaError_t e_ = cudaFuncSetAttribute(quantize_rows_kernel<BF16, CBV, E>,                       \
                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);  \
             if (e_ != cudaSuccess) return e_;                                                               \
         }                                                                                                   \
-        quantize_row32_kernel<BF16, CBV><<<grid, threads, smem, st>>>(x, rows, cols, ld, bits, had_block,   \
-                                                                      qc, S, R, codes, scales, mask, op8);  \
+        quantize_rows_kernel<BF16, CBV, E><<<grid, threads, smem, st>>>(a);                                 \
     } while (0)
     switch (cb) {
         case 1: QUEST_LAUNCH(1); break;
@@ -366,27 +397,49 @@ static cudaError_t launch_row32(int cb, dim3 grid, int threads, size_t smem, cud
 
 }  // namespace
 
-int launch_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
-                    int bits, int had_block, float trust_factor,
-                    uint8_t *codes, float *scales, uint8_t *mask, int8_t *op8, cudaStream_t st) {
-    if (rows == 0) return QUEST_OK;
+int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
+                    float trust_factor, cudaStream_t st) {
     const QuantConsts qc = make_quant_consts(bits, had_block, trust_factor);
+    const int cb = container_bits(bits);
     if (cols % 32 == 0) {
-        const int T = (int)(cols / 32);
+        const int E = (cols % 64 == 0) ? 64 : 32;
+        const int T = (int)(cols / E);
         int S;
         if (T < 32) { S = 1; while (S < T) S <<= 1; } else { S = (T + 31) / 32 * 32; }
         const int R = S >= 256 ? 1 : 256 / S;
         const int threads = R * S;
-        const int warps = threads / 32;
-        const size_t smem = had_block >= 2048 ? sizeof(float) * 32 * (size_t)threads : sizeof(float) * (size_t)warps;
-        const dim3 grid((unsigned)((rows + R - 1) / R));
-        const int cb = container_bits(bits);
-        cudaError_t e = dtype == QUEST_BF16
-            ? launch_row32<true>(cb, grid, threads, smem, st, x, rows, (int)cols, ld, bits, had_block, qc, S, R,
-                                 codes, scales, mask, op8)
-            : launch_row32<false>(cb, grid, threads, smem, st, x, rows, (int)cols, ld, bits, had_block, qc, S, R,
-                                  codes, scales, mask, op8);
-        return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+        const int warps = (threads + 31) / 32;
+        const size_t smem = had_block >= 64 * E ? sizeof(float) * E * (size_t)threads : sizeof(float) * (size_t)warps;
+        // at most two tensors per launch
+        for (int j0 = 0; j0 < njobs; j0 += 2) {
+            QuantArgs a;
+            int nb[2] = {0, 0};
+            for (int j = 0; j < 2; ++j) {
+                QuantTensor &t = a.t[j];
+                if (j0 + j < njobs) {
+                    const QuantJob &q = jobs[j0 + j];
+                    t.x = q.x; t.rows = q.rows; t.ld = q.ld; t.codes = q.codes; t.scales = q.scales;
+                    t.mask = q.mask; t.op8 = q.op8; t.rowsum = q.rowsum;
+                    nb[j] = (int)((q.rows + R - 1) / R);
+                } else {
+                    t.x = nullptr; t.rows = 0; t.ld = 0; t.codes = nullptr; t.scales = nullptr;
+                    t.mask = nullptr; t.op8 = nullptr; t.rowsum = nullptr;
+                }
+            }
+            if (nb[0] + nb[1] == 0) continue;
+            a.blocks0 = nb[0];
+            a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = S; a.R = R;
+            const dim3 grid((unsigned)(nb[0] + nb[1]));
+            cudaError_t e;
+            if (E == 64)
+                e = dtype == QUEST_BF16 ? launch_rows<true, 64>(cb, grid, threads, smem, st, a)
+                                        : launch_rows<false, 64>(cb, grid, threads, smem, st, a);
+            else
+                e = dtype == QUEST_BF16 ? launch_rows<true, 32>(cb, grid, threads, smem, st, a)
+                                        : launch_rows<false, 32>(cb, grid, threads, smem, st, a);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        return QUEST_OK;
     }
     int p2 = 1;
     while (p2 < cols) p2 <<= 1;
@@ -398,11 +451,20 @@ int launch_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_
         if (e != cudaSuccess) return cuda_fail(e);
         attr_done = true;
     }
-    const int grid = (int)(rows < 148 * 8 ? rows : 148 * 8);
-    quantize_generic_kernel<<<grid, 256, smem, st>>>(x, dtype, rows, (int)cols, ld, bits, had_block, qc, p2,
-                                                     codes, scales, mask, op8);
-    cudaError_t e = cudaGetLastError();
-    return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+    for (int j = 0; j < njobs; ++j) {
+        const QuantJob &q = jobs[j];
+        if (q.rows == 0) continue;
+        const int grid = (int)(q.rows < 148 * 8 ? q.rows : 148 * 8);
+        quantize_generic_kernel<<<grid, 256, smem, st>>>(q.x, dtype, q.rows, (int)cols, q.ld, bits, had_block, qc, p2,
+                                                         q.codes, q.scales, q.mask, q.op8);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (q.rowsum && q.op8) {
+            int s2 = launch_rowsum(q.op8, q.rows, cols, q.rowsum, st);
+            if (s2) return s2;
+        }
+    }
+    return QUEST_OK;
 }
 
 }  // namespace quest

@@ -59,7 +59,7 @@ extern "C" int quest_lowbit_gemm_static(const uint8_t *xq, const float *sx, int 
     const size_t need = quest_workspace_bytes(M, N, K, bits_x, bits_w);
     if (need == 0) {
         const int64_t worst = K * (((int64_t)1 << bits_x) - 1) * (((int64_t)1 << bits_w) - 1);
-        return (K >= 32 && K % 32 == 0 && K <= ((int64_t)1 << 24) && worst >= ((int64_t)1 << 31))
+        return (K >= 32 && K % 32 == 0 && K <= 65504 && worst >= ((int64_t)1 << 31))
                    ? QUEST_ERR_OVERFLOW : QUEST_ERR_SHAPE;
     }
     if (need > (size_t)QUEST_STATIC_SCRATCH_BYTES) return QUEST_ERR_STATIC_LIMIT;

@@ -46,7 +46,7 @@ def test_size_helpers_and_table(lib):
     ws = lib.quest_workspace_bytes(4096, 2048, 2048, 4, 4)
     assert ws >= 4096 * 2048 + 2048 * 2048 and ws % 256 == 0
     assert lib.quest_workspace_bytes(16, 16, 48, 4, 4) == 0          # K % 32 != 0
-    assert lib.quest_workspace_bytes(16, 16, 1 << 20, 8, 8) == 0     # would overflow int32
+    assert lib.quest_workspace_bytes(16, 16, 33056, 8, 8) == 0       # would overflow int32
     assert abs(lib.quest_alpha_star(1) - 0.7978846) < 1e-7
     assert abs(lib.quest_alpha_star(4) - 2.5140045) < 1e-6
     assert lib.quest_alpha_star(0) == 0.0
@@ -84,7 +84,7 @@ def test_trust_mask_requires_mask(lib):
 @pytest.mark.parametrize("kwargs,expected", [
     (dict(xq=None), 1), (dict(y=None, acc=None), 1), (dict(sx=None), 1),
     (dict(bits_x=0), 3), (dict(bits_w=12), 3), (dict(K=16), 2), (dict(K=100), 2), (dict(M=-1), 2),
-    (dict(K=1 << 20, bits_x=8, bits_w=8), 9), (dict(y_dtype=5), 5), (dict(ldy=8), 2),
+    (dict(K=33056, bits_x=8, bits_w=8), 9), (dict(K=1 << 20), 2), (dict(y_dtype=5), 5), (dict(ldy=8), 2),
     (dict(ws=None), 8), (dict(ws_bytes=16), 8), (dict(ws=ctypes.c_void_p(0x10010)), 8),
     (dict(xq=ctypes.c_void_p(0x10008)), 6),
 ])

@@ -75,10 +75,10 @@ def test_extreme_codes_do_not_overflow():
     _, acc = quest.quest_lowbit_gemm(torch.from_numpy(top).cuda(), ones[:130], 4, torch.from_numpy(bot).cuda(), ones, 4,
                                      K, want_y=False, want_acc=True)
     assert bool((acc == -K * 225).all())
-    k8 = np.full((16, 8192), 255, np.uint8)
-    with pytest.raises((quest.QuestError, ValueError)):  # K = 2^20 at 8 bits could overflow int32: refused on the host
+    k8 = np.full((16, 33056), 255, np.uint8)
+    with pytest.raises((quest.QuestError, ValueError)):  # K = 33056 at 8 bits could overflow int32: refused on the host
         quest.quest_lowbit_gemm(torch.from_numpy(k8).cuda(), ones[:16], 8, torch.from_numpy(k8).cuda(), ones[:16], 8,
-                                1 << 20)
+                                33056)
 
 
 def test_empty_product_is_a_no_op():

@@ -88,4 +88,4 @@ def test_sizes_beyond_the_static_scratch_are_refused_on_the_host():
     assert b"static scratch" in L.quest_status_string(13)
     assert call(64, 64, 48) == 2            # K not a multiple of 32: a shape error, as in quest_lowbit_gemm
     assert call(64, 64, 128, 0, 4) == 3     # bits out of range
-    assert call(16, 16, 1 << 20, 8, 8) == 9  # would overflow int32
+    assert call(16, 16, 33056, 8, 8) == 9   # would overflow int32
