@@ -10,14 +10,24 @@
 // for b = 8 (|c| up to 255) it is v = k - 128 and the epilogue restores
 // c_x . c_w = 4 v_x.v_w + 2 sum(v_x) + 2 sum(v_w) + K exactly from per-row sums.
 //
-// Kernel structure (one CTA per SM, persistent over 128 x BN output tiles):
-//   warp 0      TMA producer: 128B-swizzled K-major tiles of A (128 x 128 B) and B (BN x 128 B)
-//               into a 4-stage shared-memory ring, completion on mbarriers
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=32) x 4 per stage into
-//               one of two TMEM accumulator buffers; tcgen05.commit releases the stage / signals
-//               the epilogue
-//   warps 2..5  epilogue: tcgen05.ld 32 columns at a time, integer correction, scale, convert,
-//               store; overlaps the next tile's main loop through the second TMEM buffer
+// Two launch shapes of one kernel template.  TWO = false: one CTA per SM, persistent over 128 x BN
+// output tiles.  TWO = true: clusters of two CTAs (tcgen05 cta_group::2) persistent over 256 x 256
+// tiles; each CTA stages its own 128 rows of A and its own 128 of the tile's 256 rows of B, the
+// leader CTA issues one M=256 MMA that reads both CTAs' shared memory, and each CTA's TMEM holds
+// its 128 accumulator rows.  That cuts the operand bytes a CTA pulls from L2 per MAC by a third,
+// which is what bounds the single-CTA shape.  No TMA multicast is used: every CTA loads only tiles
+// it alone needs.
+//
+// Kernel structure:
+//   warp 0      TMA producer: 128B-swizzled K-major tiles of A (128 x 128 B) and B (BN or BN/2 rows
+//               x 128 B) into a 3..5-stage shared-memory ring, completion on mbarriers
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128 or 256, N=BN, K=32) x 4 per stage
+//               into one of two TMEM accumulator buffers; tcgen05.commit releases the stage /
+//               signals the epilogue
+//   warps 2..9  epilogue: each warp reads its 32 rows x BN/2 columns with tcgen05.ld, hands the TMEM
+//               buffer back at once, then applies the integer correction and the scales, converts,
+//               stages 32 x 128-byte slabs in shared memory and stores them with TMA tile stores;
+//               overlaps the next tile's main loop through the second TMEM buffer
 // Every wait is bounded: on expiry the CTA records a status word, stops issuing work and exits
 // through the common tail (which frees its TMEM).
 #include <cuda.h>
@@ -33,7 +43,8 @@ constexpr int BM = 128;          // tile rows (TMEM lanes)
 constexpr int BK = 128;          // bytes (= int8 elements) of K per pipeline stage: one swizzle row
 constexpr int UMMA_K = 32;       // K per tcgen05.mma kind::i8
 constexpr int STAGES = 4;
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 8;     // two per TMEM lane quarter, each taking half of the tile's columns
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
 
 enum { ST_OK = 0, ST_PRODUCER = 1, ST_MMA = 2, ST_EPILOGUE = 3 };
@@ -129,10 +140,54 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                  : "memory");
 }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// cta_group::2 forms: the load may signal an mbarrier of the peer CTA; the MMA spans both CTAs of
+// the pair; the commit arrives on the same barrier offset in every CTA named by the mask.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(cluster_bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3)
+                 : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+constexpr int MAX_STAGES = 6;
+
+// 32 columns of this warp's 32 TMEM lanes, issued without waiting: the registers are valid only
+// after tmem_wait_ld() and pin() (an empty volatile asm that makes every later use depend on a
+// statement ordered after the wait).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t *r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -143,32 +198,43 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void pin(uint32_t &v) { asm volatile("" : "+r"(v)::"memory"); }
 
-template <int BN>
+template <int BN, bool TWO>
 struct SmemLayout {
+    static constexpr int NSTAGES = TWO ? 5 : (BN == 256 ? 3 : STAGES);
     static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
+    static constexpr int B_ROWS = TWO ? BN / 2 : BN;         // rows of B this CTA stages
+    static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-    static constexpr int SW_OFFSET = BAR_OFFSET + 256;       // [2][BN] column scales
+    static constexpr int BAR_OFFSET = NSTAGES * STAGE_BYTES;
+    static constexpr int STG_OFFSET = BAR_OFFSET;            // [8 warps][32 rows x 128 B] output staging
+    static constexpr int STG_BYTES = EPI_WARPS * 4096;
+    static constexpr int BAR_OFFSET2 = STG_OFFSET + STG_BYTES;
+    static constexpr int SW_OFFSET = BAR_OFFSET2 + 256;      // [2][BN] column scales
     static constexpr int CB_OFFSET = SW_OFFSET + 2 * BN * 4; // [2][BN] column corrections (8-bit codes)
     static constexpr int TOTAL = CB_OFFSET + 2 * BN * 4 + 1024;   // + slack for 1024-byte alignment
 };
 
-template <int BN, bool CORR>
+// YT: y leaves through shared memory and TMA tile stores (whole 128-byte row segments per
+// transaction) instead of per-thread 16-byte stores, which write every 32-byte sector twice.
+template <int BN, bool CORR, bool TWO, bool YT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams p) {
-    using L = SmemLayout<BN>;
+gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmY, GemmParams p) {
+    using L = SmemLayout<BN, TWO>;
+    constexpr int STAGES = L::NSTAGES;
+    constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET);
+    uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-byte aligned, still a shared pointer
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET2);
     uint64_t *full_bar = bars;                   // [STAGES] TMA -> MMA
-    uint64_t *empty_bar = bars + STAGES;         // [STAGES] MMA -> TMA
-    uint64_t *tfull_bar = bars + 2 * STAGES;     // [2] MMA -> epilogue
-    uint64_t *tempty_bar = bars + 2 * STAGES + 2;  // [2] epilogue -> MMA
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+    uint64_t *empty_bar = bars + MAX_STAGES;     // [STAGES] MMA -> TMA
+    uint64_t *tfull_bar = bars + 2 * MAX_STAGES;     // [2] MMA -> epilogue
+    uint64_t *tempty_bar = bars + 2 * MAX_STAGES + 2;  // [2] epilogue -> MMA
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     float *sw_tile = reinterpret_cast<float *>(smem + L::SW_OFFSET);
     int32_t *cb_tile = reinterpret_cast<int32_t *>(smem + L::CB_OFFSET);
@@ -176,6 +242,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     constexpr uint32_t TMEM_COLS = 2 * BN;       // two accumulator buffers
+    // pair variant: rank of this CTA in its cluster of two; rank 0 leads (issues the MMAs, owns the
+    // full and accumulator-empty barriers that both CTAs signal)
+    const uint32_t rank = TWO ? cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
+    const int unit = TWO ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;          // tile-loop index
+    const int num_units = TWO ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -184,24 +256,32 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tfull_bar[b]), 1);
-            mbar_init(smem_u32(&tempty_bar[b]), 4);
+            mbar_init(smem_u32(&tempty_bar[b]), TWO ? 2 * EPI_WARPS : EPI_WARPS);   // epilogue warps (of both CTAs of a pair)
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // barriers visible to the TMA unit
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (TWO) {      // executed by this warp of both CTAs of the pair
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                         "r"(TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                         "r"(TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (TWO) cluster_sync_all();       // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int num_m = (p.M + BM - 1) / BM;
+    const int num_m = (p.M + TILE_M - 1) / TILE_M;
     const int num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
@@ -211,17 +291,25 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % num_m) * BM;
-                const int n0 = (tile / num_m) * BN;
+            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+                const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;          // this CTA's rows of A
+                const int n0 = (tile / num_m) * BN + (int)rank * L::B_ROWS;      // this CTA's rows of B
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, p.status, ST_PRODUCER);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(&full_bar[stage]);
-                    mbar_expect_tx(fb, L::STAGE_BYTES);
                     uint8_t *sa = smem + stage * L::STAGE_BYTES;
-                    tma_load_2d(smem_u32(sa), &tmA, kb * BK, m0, fb);
-                    tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
+                    if constexpr (TWO) {
+                        // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
+                        if (leader) mbar_expect_tx(fb, 2 * L::STAGE_BYTES);
+                        const uint32_t lfb = mapa_shared(fb, 0);
+                        tma_load_2d_pair(smem_u32(sa), &tmA, kb * BK, m0, lfb);
+                        tma_load_2d_pair(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, lfb);
+                    } else {
+                        mbar_expect_tx(fb, L::STAGE_BYTES);
+                        tma_load_2d(smem_u32(sa), &tmA, kb * BK, m0, fb);
+                        tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
+                    }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -235,13 +323,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_i8(BM, BN);
+        if (lane == 0 && leader) {
+            constexpr uint32_t idesc = make_idesc_i8(TILE_M, BN);
             int stage = 0;
             uint32_t phase = 0;
             int t = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+            for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
                 const int buf = t & 1;
                 const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
                 ok = mbar_wait(smem_u32(&tempty_bar[buf]), bphase ^ 1u, abort_flag, p.status, ST_MMA);
@@ -258,27 +346,41 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int kk = 0; kk < BK / UMMA_K; ++kk) {
                         // advance along K inside the 128-byte swizzle row: +32 bytes = +2 in 16-byte units
-                        umma_i8(d_tmem, a_desc + (uint64_t)(kk * (UMMA_K >> 4)), b_desc + (uint64_t)(kk * (UMMA_K >> 4)),
-                                idesc, (kb | kk) != 0 ? 1u : 0u);
+                        if constexpr (TWO)
+                            umma_i8_pair(d_tmem, a_desc + (uint64_t)(kk * (UMMA_K >> 4)),
+                                         b_desc + (uint64_t)(kk * (UMMA_K >> 4)), idesc, (kb | kk) != 0 ? 1u : 0u);
+                        else
+                            umma_i8(d_tmem, a_desc + (uint64_t)(kk * (UMMA_K >> 4)),
+                                    b_desc + (uint64_t)(kk * (UMMA_K >> 4)), idesc, (kb | kk) != 0 ? 1u : 0u);
                     }
-                    umma_commit(smem_u32(&empty_bar[stage]));     // stage reusable once these MMAs retire
+                    // stage reusable (in both CTAs of a pair) once these MMAs retire
+                    if constexpr (TWO) umma_commit_pair(smem_u32(&empty_bar[stage]));
+                    else umma_commit(smem_u32(&empty_bar[stage]));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) umma_commit(smem_u32(&tfull_bar[buf]));   // accumulator complete
+                if (ok) {                                          // accumulator complete
+                    if constexpr (TWO) umma_commit_pair(smem_u32(&tfull_bar[buf]));
+                    else umma_commit(smem_u32(&tfull_bar[buf]));
+                }
             }
         }
         __syncwarp();
     } else {
-        // ---- epilogue: 4 warps, warp q reads TMEM lanes [32q, 32q+32) = tile rows 32q + lane ----
+        // ---- epilogue: 8 warps; warp w reads TMEM lanes [32 (w & 3), +32) = tile rows 32 (w & 3) + lane
+        //      and the column half (w - 2) / 4 of the tile ------------------------------------------------
+        constexpr int CW = BN / 2;                     // columns per warp
         const int quarter = warp & 3;
-        const int ep_tid = threadIdx.x - 64;           // 0..127 over the epilogue warps
+        const int cbase = ((warp - 2) >> 2) * CW;
+        const int ep_tid = threadIdx.x - 64;           // 0..255 over the epilogue warps
         int t = 0;
         bool ok = true;
         const bool vec_y = p.y && (((reinterpret_cast<uintptr_t>(p.y) & 15) == 0) &&
                                    (p.ldy % (p.y_dtype == QUEST_BF16 ? 8 : 4) == 0));
         const bool vec_acc = p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
-            const int m0 = (tile % num_m) * BM;
+        const bool y_f32 = p.y_dtype == QUEST_F32;
+        uint8_t *slab = smem + L::STG_OFFSET + (warp - 2) * 4096;
+        for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
+            const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
             const int n0 = (tile / num_m) * BN;
             const int buf = t & 1;
             const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
@@ -287,114 +389,186 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // arrived at the barrier of tile t-1
             float *swt = sw_tile + buf * BN;
             int32_t *cbt = cb_tile + buf * BN;
-            for (int c = ep_tid; c < BN; c += 128) {
+            for (int c = ep_tid; c < BN; c += 32 * EPI_WARPS) {
                 const int col = n0 + c;
                 swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
                 if (CORR) cbt[c] = (p.rs_b && col < p.N) ? p.cb * __ldg(p.rs_b + col) : 0;
             }
+            const int row = m0 + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+            const float sxr = (row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
+            int rsa = 0;
+            if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
             ok = mbar_wait(smem_u32(&tfull_bar[buf]), bphase, abort_flag, p.status, ST_EPILOGUE);
-            // one barrier over the 128 epilogue threads publishes the staged scales and makes the
+            // one barrier over the epilogue threads publishes the staged scales and makes the
             // continue/abort decision unanimous, so no warp can be left waiting at a later barrier
             {
                 uint32_t all_ok;
                 asm volatile(
                     "{\n\t.reg .pred p, q;\n\t"
                     "setp.ne.u32 q, %1, 0;\n\t"
-                    "bar.red.and.pred p, 1, 128, q;\n\t"
+                    "bar.red.and.pred p, 1, %2, q;\n\t"
                     "selp.u32 %0, 1, 0, p;\n\t}"
                     : "=r"(all_ok)
-                    : "r"((uint32_t)(ok ? 1u : 0u))
+                    : "r"((uint32_t)(ok ? 1u : 0u)), "n"(32 * EPI_WARPS)
                     : "memory");
                 ok = all_ok != 0;
             }
             if (!ok) break;
             tc_fence_after();
-            const int row = m0 + quarter * 32 + lane;
-            const bool row_ok = row < p.M;
-            const float sxr = (row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
-            int rsa = 0;
-            if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= p.N) break;             // uniform across the CTA
-                uint32_t r[32];
-                tmem_ld32(t_row + (uint32_t)c0, r);
-                if (!row_ok) continue;
-                const int col0 = n0 + c0;
-                const bool full = col0 + 32 <= p.N;
-                if (CORR) {
+            // all of this warp's accumulator columns in one go, then hand the TMEM buffer back to
+            // the MMA warp before any arithmetic
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cbase);
+            uint32_t r[CW];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        r[j] = (uint32_t)((int32_t)((uint32_t)p.mul * r[j] + (uint32_t)rsa + (uint32_t)cbt[c0 + j]) >> p.sh);
-                } else {
+            for (int c0 = 0; c0 < CW; c0 += 32)
+                if (n0 + cbase + c0 < p.N) tmem_ld32_issue(t_row + (uint32_t)c0, &r[c0]);     // uniform predicate
+            tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = (uint32_t)((int32_t)r[j] >> p.sh);
-                }
-                if (p.acc) {
-                    int32_t *dst = p.acc + (long long)row * p.N + col0;
-                    if (vec_acc && full) {
+            for (int j = 0; j < CW; ++j) pin(r[j]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if constexpr (TWO) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[buf]), 0));   // the leader's barrier
+                else mbar_arrive(smem_u32(&tempty_bar[buf]));
+            }
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<uint4 *>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-                    } else {
+            for (int c0 = 0; c0 < CW; c0 += 32) {
+                const int col0 = n0 + cbase + c0;
+                if (col0 < p.N) {                      // uniform across the warp
+                    const bool full = col0 + 32 <= p.N;
+                    uint32_t *rc = &r[c0];
+                    if (CORR) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) dst[j] = (int32_t)r[j];
-                    }
-                }
-                if (p.y) {
-                    // y = (sx * sw) * acc, each product rounded to binary32
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        r[j] = __float_as_uint(__fmul_rn(__fmul_rn(sxr, swt[c0 + j]), (float)(int32_t)r[j]));
-                    if (p.y_dtype == QUEST_BF16) {
-                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.y) + (long long)row * p.ldy + col0;
-                        if (vec_y && full) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                uint4 q;
-                                __nv_bfloat162 h;
-                                h = __floats2bfloat162_rn(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-                                q.x = *reinterpret_cast<uint32_t *>(&h);
-                                h = __floats2bfloat162_rn(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                                q.y = *reinterpret_cast<uint32_t *>(&h);
-                                h = __floats2bfloat162_rn(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
-                                q.z = *reinterpret_cast<uint32_t *>(&h);
-                                h = __floats2bfloat162_rn(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
-                                q.w = *reinterpret_cast<uint32_t *>(&h);
-                                *reinterpret_cast<uint4 *>(dst + j) = q;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
-                        }
+                            rc[j] = (uint32_t)((int32_t)((uint32_t)p.mul * rc[j] + (uint32_t)rsa +
+                                                         (uint32_t)cbt[cbase + c0 + j]) >> p.sh);
                     } else {
-                        float *dst = reinterpret_cast<float *>(p.y) + (long long)row * p.ldy + col0;
-                        if (vec_y && full) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) rc[j] = (uint32_t)((int32_t)rc[j] >> p.sh);
+                    }
+                    if (p.acc && row_ok) {
+                        int32_t *dst = p.acc + (long long)row * p.N + col0;
+                        if (vec_acc && full) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(rc[j], rc[j + 1], rc[j + 2], rc[j + 3]);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]);
+                                if (col0 + j < p.N) dst[j] = (int32_t)rc[j];
+                        }
+                    }
+                    if (p.y) {
+                        // y = (sx * sw) * acc, each product rounded to binary32
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            rc[j] = __float_as_uint(__fmul_rn(__fmul_rn(sxr, swt[cbase + c0 + j]), (float)(int32_t)rc[j]));
+                        if constexpr (YT) {
+                            // stage 32 rows x 128 bytes (128-byte swizzle: 16-byte chunk j of row r sits at
+                            // j ^ (r & 7)), then one lane stores the slab with a TMA tile store, which clips
+                            // at the matrix edges.  Binary32 fills a slab per 32 columns, bfloat16 per 64.
+                            const int half = y_f32 ? 0 : ((c0 >> 5) & 1);
+                            if (half == 0) {
+                                // the previous store from this slab must have finished reading it
+                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                                __syncwarp();
+                            }
+                            uint8_t *rowp = slab + lane * 128;
+                            const int sw7 = lane & 7;
+                            if (y_f32) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    *reinterpret_cast<uint4 *>(rowp + ((j ^ sw7) << 4)) =
+                                        make_uint4(rc[4 * j], rc[4 * j + 1], rc[4 * j + 2], rc[4 * j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    uint4 q;
+                                    __nv_bfloat162 h;
+                                    h = __floats2bfloat162_rn(__uint_as_float(rc[8 * j]), __uint_as_float(rc[8 * j + 1]));
+                                    q.x = *reinterpret_cast<uint32_t *>(&h);
+                                    h = __floats2bfloat162_rn(__uint_as_float(rc[8 * j + 2]), __uint_as_float(rc[8 * j + 3]));
+                                    q.y = *reinterpret_cast<uint32_t *>(&h);
+                                    h = __floats2bfloat162_rn(__uint_as_float(rc[8 * j + 4]), __uint_as_float(rc[8 * j + 5]));
+                                    q.z = *reinterpret_cast<uint32_t *>(&h);
+                                    h = __floats2bfloat162_rn(__uint_as_float(rc[8 * j + 6]), __uint_as_float(rc[8 * j + 7]));
+                                    q.w = *reinterpret_cast<uint32_t *>(&h);
+                                    *reinterpret_cast<uint4 *>(rowp + (((half * 4 + j) ^ sw7) << 4)) = q;
+                                }
+                            }
+                            const bool flush = y_f32 || half == 1 || (col0 + 32 >= p.N);
+                            if (flush) {
+                                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                                __syncwarp();
+                                if (lane == 0) {
+                                    const int first_col = y_f32 ? col0 : col0 - half * 32;
+                                    const int xbytes = first_col * (y_f32 ? 4 : 2);       // a multiple of 64
+                                    asm volatile(
+                                        "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                        ::"l"(reinterpret_cast<uint64_t>(&tmY)), "r"(smem_u32(slab)), "r"(xbytes),
+                                          "r"(m0 + quarter * 32)
+                                        : "memory");
+                                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                                }
+                            }
+                        } else if (row_ok) {
+                            if (p.y_dtype == QUEST_BF16) {
+                                __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.y) + (long long)row * p.ldy + col0;
+                                if (vec_y && full) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 8) {
+                                        uint4 q;
+                                        __nv_bfloat162 h;
+                                        h = __floats2bfloat162_rn(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]));
+                                        q.x = *reinterpret_cast<uint32_t *>(&h);
+                                        h = __floats2bfloat162_rn(__uint_as_float(rc[j + 2]), __uint_as_float(rc[j + 3]));
+                                        q.y = *reinterpret_cast<uint32_t *>(&h);
+                                        h = __floats2bfloat162_rn(__uint_as_float(rc[j + 4]), __uint_as_float(rc[j + 5]));
+                                        q.z = *reinterpret_cast<uint32_t *>(&h);
+                                        h = __floats2bfloat162_rn(__uint_as_float(rc[j + 6]), __uint_as_float(rc[j + 7]));
+                                        q.w = *reinterpret_cast<uint32_t *>(&h);
+                                        *reinterpret_cast<uint4 *>(dst + j) = q;
+                                    }
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j)
+                                        if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(rc[j]));
+                                }
+                            } else {
+                                float *dst = reinterpret_cast<float *>(p.y) + (long long)row * p.ldy + col0;
+                                if (vec_y && full) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 4)
+                                        *reinterpret_cast<uint4 *>(dst + j) = make_uint4(rc[j], rc[j + 1], rc[j + 2], rc[j + 3]);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j)
+                                        if (col0 + j < p.N) dst[j] = __uint_as_float(rc[j]);
+                                }
+                            }
                         }
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
         }
     }
 
+    if constexpr (YT) {
+        // output tiles still on their way out of shared memory
+        if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
     tc_fence_before();
     __syncthreads();
+    // a CTA of a pair must stay until its peer can no longer signal its barriers or read its
+    // shared memory and tensor memory
+    if constexpr (TWO) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        if constexpr (TWO)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -466,22 +640,55 @@ int make_operand_map(CUtensorMap *tm, const int8_t *base, int64_t rows, int64_t 
     return QUEST_OK;
 }
 
-template <int BN, bool CORR>
-int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmParams &p, cudaStream_t st) {
+// y viewed as bytes: [rows x row_bytes], row pitch pitch_bytes; box = 128 bytes x 32 rows, 128-byte swizzle.
+int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes, int64_t pitch_bytes) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return cuda_fail_msg("cuTensorMapEncodeTiled entry point not available");
+    cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch_bytes};
+    cuuint32_t box[2] = {128, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail_msg("cuTensorMapEncodeTiled failed for the output");
+    return QUEST_OK;
+}
+
+template <int BN, bool CORR, bool TWO, bool YT>
+int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
+                   cudaStream_t st) {
+    using L = SmemLayout<BN, TWO>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, CORR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SmemLayout<BN>::TOTAL);
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, CORR, TWO, YT>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
         attr_done = true;
     }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int tiles = ((p.M + BM - 1) / BM) * ((p.N + BN - 1) / BN);
-    const int grid = tiles < sms ? tiles : sms;
-    gemm_i8_kernel<BN, CORR><<<grid, NUM_THREADS, SmemLayout<BN>::TOTAL, st>>>(tmA, tmB, p);
-    cudaError_t e = cudaGetLastError();
+    const int tile_m = TWO ? 2 * BM : BM;
+    const int tiles = ((p.M + tile_m - 1) / tile_m) * ((p.N + BN - 1) / BN);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    if (TWO) {
+        const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+        cfg.gridDim = dim3((unsigned)(2 * pairs));
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    } else {
+        cfg.gridDim = dim3((unsigned)(tiles < sms ? tiles : sms));
+    }
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = L::TOTAL;
+    cfg.stream = st;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<BN, CORR, TWO, YT>, tmA, tmB, tmY, p);
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
 
@@ -551,14 +758,30 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
     if (!p.status) return QUEST_ERR_CUDA;
 
     const bool wide = N > 128;
+    const bool pair = wide && M > 128;             // 256 x 256 tiles on CTA pairs
     CUtensorMap tmA, tmB;
     int s = make_operand_map(&tmA, a8, M, K, BM);
     if (s) return s;
-    s = make_operand_map(&tmB, b8, N, K, wide ? 256 : 128);
+    s = make_operand_map(&tmB, b8, N, K, pair ? 128 : wide ? 256 : 128);
     if (s) return s;
     const bool corr = (bits_x == 8) || (bits_w == 8);
-    if (wide) return corr ? launch_gemm_bn<256, true>(tmA, tmB, p, st) : launch_gemm_bn<256, false>(tmA, tmB, p, st);
-    return corr ? launch_gemm_bn<128, true>(tmA, tmB, p, st) : launch_gemm_bn<128, false>(tmA, tmB, p, st);
+    // y through TMA tile stores when its base and row pitch allow it (16-byte multiples)
+    const size_t esz = y_dtype == QUEST_F32 ? 4 : 2;
+    const bool yt = y && (reinterpret_cast<uintptr_t>(y) % 16 == 0) && ((size_t)ldy * esz % 16 == 0);
+    CUtensorMap tmY = tmA;                               // placeholder when unused
+    if (yt) {
+        s = make_output_map(&tmY, y, M, (int64_t)N * (int64_t)esz, (int64_t)ldy * (int64_t)esz);
+        if (s) return s;
+    }
+#define QUEST_GEMM(BNV, TWOV)                                                                        \
+    (corr ? (yt ? launch_gemm_bn<BNV, true, TWOV, true>(tmA, tmB, tmY, p, st)                         \
+                : launch_gemm_bn<BNV, true, TWOV, false>(tmA, tmB, tmY, p, st))                        \
+          : (yt ? launch_gemm_bn<BNV, false, TWOV, true>(tmA, tmB, tmY, p, st)                        \
+                : launch_gemm_bn<BNV, false, TWOV, false>(tmA, tmB, tmY, p, st)))
+    if (pair) return QUEST_GEMM(256, true);
+    if (wide) return QUEST_GEMM(256, false);
+    return QUEST_GEMM(128, false);
+#undef QUEST_GEMM
 }
 
 }  // namespace quest
