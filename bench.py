@@ -309,15 +309,23 @@ def run_gpu(args, rank: int, world: int, local: int):
     max_elapsed = max_over_ranks(elapsed_s, world, dev)
     value = aggregate_tokens_per_s(M, args.steps, world, max_elapsed)
 
-    # ---- per-kernel durations: same loop, stages bracketed by CUDA events on the same stream
+    # ---- per-kernel durations: the same steps with every stage bracketed by CUDA events on the
+    # launching stream.  With a graph the event records are graph nodes, so the host's launch
+    # rate does not sit between an event and its kernel; each replay yields the stage times of
+    # the graph's last step.
     quest.quest_stage_timing(True)
-    quest.quest_stage_times(reset=True)
-    prof_steps = min(args.steps, 200)
-    for i in range(prof_steps):
-        step(i)
+    quest.quest_stage_times(reset=2)
+    staged = capture(step)
+    prof_reps = 50
+    for r in range(prof_reps):
+        if staged is None:
+            step(r)
+        else:
+            staged.replay()
         quest.quest_stage_times()
-    stage = quest.quest_stage_times(reset=True)
+    stage = quest.quest_stage_times(reset=2)
     quest.quest_stage_timing(False)
+    del staged
     stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
 
     # ---- end to end: pinned host inputs in, result out, every step ---------------------

@@ -184,8 +184,11 @@ int quest_device_status(void *stream);
  * quest_stage_times waits for the events of the most recent call, adds their elapsed times to
  * running totals, copies totals (milliseconds) and counts into the caller's HOST arrays of
  * QUEST_NUM_STAGES entries (either may be NULL), and zeroes the totals if reset != 0.  Call it
- * after every timed call: events are reused from call to call.  Not thread-safe; leave it
- * disabled (the default) in production.
+ * after every timed call: events are reused from call to call.  A call made while its stream is
+ * being captured records its events as graph nodes instead: every replay of the graph re-times
+ * the stages, and quest_stage_times, called after a replay, collects the stages of the LAST call
+ * in the graph (until reset == 2 forgets the captured stages).  Not thread-safe; leave it disabled
+ * (the default) in production.
  */
 enum {
     QUEST_STAGE_QUANT_X = 0,   /* quantizer launch on x (or the only launch of quest_quantize) */

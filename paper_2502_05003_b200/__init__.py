@@ -63,11 +63,13 @@ def quest_stage_timing(enable: bool) -> None:
     _lib.check(_lib.load().quest_stage_timing(1 if enable else 0))
 
 
-def quest_stage_times(reset: bool = False) -> dict:
-    """Collects the events of the latest call; returns {stage: (total_ms, count)}."""
+def quest_stage_times(reset=False) -> dict:
+    """Collects the events of the latest call (or, for calls captured into a CUDA graph, of the
+    latest replay); returns {stage: (total_ms, count)}.  ``reset``: False/0 keep the totals,
+    True/1 zero them, 2 also forget stages recorded inside a capture."""
     tot = (ctypes.c_double * len(STAGES))()
     cnt = (ctypes.c_longlong * len(STAGES))()
-    _lib.check(_lib.load().quest_stage_times(tot, cnt, 1 if reset else 0))
+    _lib.check(_lib.load().quest_stage_times(tot, cnt, int(reset)))
     return {name: (float(tot[i]), int(cnt[i])) for i, name in enumerate(STAGES)}
 
 

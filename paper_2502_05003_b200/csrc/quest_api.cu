@@ -59,6 +59,7 @@ struct StageTimer {
     cudaEvent_t ev[QUEST_NUM_STAGES][2] = {};
     bool created = false;
     bool pending[QUEST_NUM_STAGES] = {};
+    bool captured[QUEST_NUM_STAGES] = {};      // recorded inside a stream capture: re-recorded at every graph replay
     double total_ms[QUEST_NUM_STAGES] = {};
     long long count[QUEST_NUM_STAGES] = {};
 };
@@ -68,13 +69,24 @@ struct StageScope {
     int id;
     cudaStream_t st;
     bool on;
+    bool capturing = false;
     StageScope(int id_, cudaStream_t st_) : id(id_), st(st_), on(g_timer.enabled && g_timer.created) {
-        if (on) cudaEventRecord(g_timer.ev[id][0], st);
+        if (on) {
+            cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+            capturing = cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusActive;
+            record(g_timer.ev[id][0]);
+        }
+    }
+    void record(cudaEvent_t ev) {
+        // inside a capture the record becomes a graph node that times every replay
+        if (capturing) cudaEventRecordWithFlags(ev, st, cudaEventRecordExternal);
+        else cudaEventRecord(ev, st);
     }
     ~StageScope() {
         if (on) {
-            cudaEventRecord(g_timer.ev[id][1], st);
-            g_timer.pending[id] = true;
+            record(g_timer.ev[id][1]);
+            if (capturing) g_timer.captured[id] = true;
+            else g_timer.pending[id] = true;
         }
     }
 };
@@ -181,7 +193,7 @@ int quest_stage_timing(int enable) {
 
 int quest_stage_times(double *total_ms, long long *counts, int reset) {
     for (int i = 0; i < QUEST_NUM_STAGES; ++i) {
-        if (g_timer.pending[i]) {
+        if (g_timer.pending[i] || g_timer.captured[i]) {
             cudaError_t e = cudaEventSynchronize(g_timer.ev[i][1]);
             float ms = 0.0f;
             if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, g_timer.ev[i][0], g_timer.ev[i][1]);
@@ -196,6 +208,7 @@ int quest_stage_times(double *total_ms, long long *counts, int reset) {
             g_timer.total_ms[i] = 0.0;
             g_timer.count[i] = 0;
         }
+        if (reset > 1) g_timer.captured[i] = false;
     }
     return QUEST_OK;
 }

@@ -246,6 +246,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // full and accumulator-empty barriers that both CTAs signal)
     const uint32_t rank = TWO ? cluster_ctarank() : 0u;
     const bool leader = rank == 0;
+    pdl_launch_dependents();
     const int unit = TWO ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;          // tile-loop index
     const int num_units = TWO ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
@@ -280,6 +281,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if constexpr (TWO) cluster_sync_all();       // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();     // set-up above overlaps the previous kernel; operands and outputs are touched only from here
 
     const int num_m = (p.M + TILE_M - 1) / TILE_M;
     const int num_n = (p.N + BN - 1) / BN;
@@ -579,6 +581,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 template <int CB>
 __global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits, long long n_groups,
                                     int8_t *__restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n_groups;
          g += (long long)gridDim.x * blockDim.x) {
         const uint32_t *src = reinterpret_cast<const uint32_t *>(codes) + g * CB;
@@ -595,6 +599,8 @@ __global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits,
 
 // Row sums of an int8 matrix [rows x K]: one warp per row.
 __global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, int K, int32_t *__restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long row = blockIdx.x * (long long)(blockDim.x >> 5) + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -670,25 +676,15 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tile_m = TWO ? 2 * BM : BM;
     const int tiles = ((p.M + tile_m - 1) / tile_m) * ((p.N + BN - 1) / BN);
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    int grid;
     if (TWO) {
         const int pairs = tiles < sms / 2 ? tiles : sms / 2;
-        cfg.gridDim = dim3((unsigned)(2 * pairs));
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        grid = 2 * pairs;
     } else {
-        cfg.gridDim = dim3((unsigned)(tiles < sms ? tiles : sms));
+        grid = tiles < sms ? tiles : sms;
     }
-    cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = L::TOTAL;
-    cfg.stream = st;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<BN, CORR, TWO, YT>, tmA, tmB, tmY, p);
-    if (e == cudaSuccess) e = cudaGetLastError();
+    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, CORR, TWO, YT>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
+                               TWO ? 2 : 1, tmA, tmB, tmY, p);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
 
@@ -717,13 +713,13 @@ int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_
     const int threads = 256;
     long long blocks = (n_groups + threads - 1) / threads;
     if (blocks > 148 * 16) blocks = 148 * 16;
+    cudaError_t e;
     switch (container_bits(bits)) {
-        case 1: unpack_codes_kernel<1><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
-        case 2: unpack_codes_kernel<2><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
-        case 4: unpack_codes_kernel<4><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
-        default: unpack_codes_kernel<8><<<(int)blocks, threads, 0, st>>>(codes, bits, n_groups, out); break;
+        case 1: e = launch_pdl(unpack_codes_kernel<1>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
+        case 2: e = launch_pdl(unpack_codes_kernel<2>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
+        case 4: e = launch_pdl(unpack_codes_kernel<4>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
+        default: e = launch_pdl(unpack_codes_kernel<8>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
     }
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e);
     if (rowsum) return launch_rowsum(out, rows, K, rowsum, st);
     return QUEST_OK;
@@ -732,8 +728,7 @@ int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st) {
     if (rows == 0) return QUEST_OK;
     const long long rb = (rows + 7) / 8;
-    rowsum_i8_kernel<<<(int)rb, 256, 0, st>>>(a8, rows, (int)K, rowsum);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(rowsum_i8_kernel, dim3((unsigned)rb), dim3(256), 0, st, 1, a8, (long long)rows, (int)K, rowsum);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
 

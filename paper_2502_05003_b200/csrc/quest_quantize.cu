@@ -52,6 +52,8 @@ quantize_generic_kernel(const void *__restrict__ x, int dtype, int64_t rows, int
                         uint8_t *__restrict__ codes, float *__restrict__ scales,
                         uint8_t *__restrict__ mask, int8_t *__restrict__ op8) {
     extern __shared__ float smem_f[];
+    pdl_launch_dependents();
+    pdl_wait();
     float *u = smem_f;
     float *tmp = smem_f + cols;
     __shared__ float s_inv;
@@ -159,6 +161,8 @@ __global__ void __launch_bounds__(E == 64 ? 256 : 512)
 quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
     extern __shared__ float xsm[];                 // [E][blockDim.x] exchange, then [warps] partial sums
     constexpr int H = E / 2;                       // float2 pairs per thread
+    pdl_launch_dependents();
+    pdl_wait();
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int nthreads = blockDim.x;
@@ -383,7 +387,8 @@ static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cuda
                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);  \
             if (e_ != cudaSuccess) return e_;                                                               \
         }                                                                                                   \
-        quantize_rows_kernel<BF16, CBV, E><<<grid, threads, smem, st>>>(a);                                 \
+        cudaError_t l_ = launch_pdl(quantize_rows_kernel<BF16, CBV, E>, grid, dim3(threads), smem, st, 1, a);  \
+        if (l_ != cudaSuccess) return l_;                                                                   \
     } while (0)
     switch (cb) {
         case 1: QUEST_LAUNCH(1); break;
@@ -455,9 +460,8 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
         const QuantJob &q = jobs[j];
         if (q.rows == 0) continue;
         const int grid = (int)(q.rows < 148 * 8 ? q.rows : 148 * 8);
-        quantize_generic_kernel<<<grid, 256, smem, st>>>(q.x, dtype, q.rows, (int)cols, q.ld, bits, had_block, qc, p2,
-                                                         q.codes, q.scales, q.mask, q.op8);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_pdl(quantize_generic_kernel, dim3(grid), dim3(256), smem, st, 1, q.x, dtype, q.rows, (int)cols,
+                                   q.ld, bits, had_block, qc, p2, q.codes, q.scales, q.mask, q.op8);
         if (e != cudaSuccess) return cuda_fail(e);
         if (q.rowsum && q.op8) {
             int s2 = launch_rowsum(q.op8, q.rows, cols, q.rowsum, st);
