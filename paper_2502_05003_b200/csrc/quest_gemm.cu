@@ -155,7 +155,7 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // cta_group::2 forms: the load may signal an mbarrier of the peer CTA; the MMA spans both CTAs of
 // the pair; the commit arrives on the same barrier offset in every CTA named by the mask.
@@ -398,7 +398,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             const int row = m0 + quarter * 32 + lane;
             const bool row_ok = row < p.M;
-            const float sxr = (row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
+            // without 8-bit corrections and without the raw accumulators, the exact power of two of the
+            // operand scaling is folded into the row scale instead of shifting every accumulator
+            const bool fold = !CORR && !p.acc;
+            float sxr = (row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
+            if (fold) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.sh) << 23));
             int rsa = 0;
             if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
             ok = mbar_wait(smem_u32(&tfull_bar[buf]), bphase, abort_flag, p.status, ST_EPILOGUE);
@@ -445,7 +449,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int j = 0; j < 32; ++j)
                             rc[j] = (uint32_t)((int32_t)((uint32_t)p.mul * rc[j] + (uint32_t)rsa +
                                                          (uint32_t)cbt[cbase + c0 + j]) >> p.sh);
-                    } else {
+                    } else if (!fold) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) rc[j] = (uint32_t)((int32_t)rc[j] >> p.sh);
                     }
@@ -462,10 +466,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                     if (p.y) {
-                        // y = (sx * sw) * acc, each product rounded to binary32
+                        // y = (sx * sw) * acc, each product rounded to binary32 (two columns per instruction)
+                        const float2 sx2 = make_float2(sxr, sxr);
+                        const float2 *sw2 = reinterpret_cast<const float2 *>(swt + cbase + c0);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            rc[j] = __float_as_uint(__fmul_rn(__fmul_rn(sxr, swt[cbase + c0 + j]), (float)(int32_t)rc[j]));
+                        for (int j = 0; j < 32; j += 2) {
+                            const float2 a2 = make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
+                            const float2 y2 = __fmul2_rn(__fmul2_rn(sx2, sw2[j >> 1]), a2);
+                            rc[j] = __float_as_uint(y2.x);
+                            rc[j + 1] = __float_as_uint(y2.y);
+                        }
                         if constexpr (YT) {
                             // stage 32 rows x 128 bytes (128-byte swizzle: 16-byte chunk j of row r sits at
                             // j ^ (r & 7)), then one lane stores the slab with a TMA tile store, which clips
