@@ -156,57 +156,23 @@ struct QuantArgs {
     int S, R;
 };
 
-template <bool BF16, int CB, int E>
-__global__ void __launch_bounds__(E == 64 ? 256 : 512)
-quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
-    extern __shared__ float xsm[];                 // [E][blockDim.x] exchange, then [warps] partial sums
-    constexpr int H = E / 2;                       // float2 pairs per thread
-    pdl_launch_dependents();
-    pdl_wait();
+// Everything after the load: rotation from stride s_start downwards (larger strides already
+// applied by the caller), RMS, projection, trust test, packing and stores for the E elements this
+// thread holds.  GFULL: had_block >= E, so every in-register stage runs.
+template <int CB, int E, bool GFULL>
+__device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
+                                                     bool active, long long row, int tr, int r_local, float *xsm,
+                                                     int s_start) {
+    constexpr int H = E / 2;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int nthreads = blockDim.x;
-    const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
-    const QuantTensor &tn = a.t[which];
-    const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
     const int S = a.S;
-    const int r_local = tid / S;
-    const int tr = tid - r_local * S;              // slot inside the row
-    const long long row = (long long)blk * a.R + r_local;
     const int cols = a.cols;
     const int had_block = a.had_block;
-    const int T = cols / E;
-    const bool active = (row < tn.rows) && (tr < T);
-
-    float2 v[H];
-    if (active) {
-        if (BF16) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(tn.x) + row * tn.ld + (long long)tr * E);
-#pragma unroll
-            for (int q = 0; q < E / 8; ++q) {
-                const uint4 w = __ldg(src + q);
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    v[q * 4 + j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
-            }
-        } else {
-            const float4 *src = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(tn.x) + row * tn.ld + (long long)tr * E);
-#pragma unroll
-            for (int q = 0; q < E / 4; ++q) {
-                const float4 w = __ldg(src + q);
-                v[q * 2] = make_float2(w.x, w.y);
-                v[q * 2 + 1] = make_float2(w.z, w.w);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
-    }
-
     // ---- rotation, descending stride --------------------------------------------------------
     const float2 neg1 = make_float2(-1.0f, -1.0f);
-    for (int s = had_block >> 1; s >= 32 * E; s >>= 1) {      // partner thread is in another warp
+    for (int s = s_start; s >= 32 * E; s >>= 1) {             // partner thread is in another warp
         const int dist = s / E;
         float2 *x2 = reinterpret_cast<float2 *>(xsm);
         __syncthreads();
@@ -220,7 +186,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
         for (int i = 0; i < H; ++i) v[i] = __ffma2_rn(v[i], sgn, x2[i * nthreads + pt]);
     }
     {
-        int s0 = had_block >> 1;
+        int s0 = s_start;
         if (s0 > 16 * E) s0 = 16 * E;
 #pragma unroll 1
         for (int s = s0; s >= E; s >>= 1) {                    // partner thread is a lane of this warp
@@ -238,7 +204,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
     }
 #pragma unroll
     for (int s = E / 2; s >= 2; s >>= 1) {                     // partner element is in this thread
-        if (s < had_block) {
+        if (GFULL || s < had_block) {
             const int s2 = s >> 1;
 #pragma unroll
             for (int i = 0; i < H; ++i)
@@ -249,7 +215,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
                 }
         }
     }
-    if (had_block > 1) {
+    if (GFULL || had_block > 1) {
 #pragma unroll
         for (int i = 0; i < H; ++i) {
             const float p = v[i].x, q = v[i].y;
@@ -288,7 +254,6 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
     }
     const float rms = __fsqrt_rn(__fdiv_rn(ss, (float)cols));
     const float inv = (rms > 0.0f) ? __fdiv_rn(a.qc.A, rms) : 0.0f;
-    if (!active && tn.rowsum == nullptr) return;
     if (active && tn.scales && tr == 0) tn.scales[row] = __fmul_rn(rms, a.qc.B);
 
     // ---- project: level axis, clamp, round to nearest even, trust test -----------------------
@@ -378,6 +343,150 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
     }
 }
 
+template <bool BF16, int CB, int E>
+__global__ void __launch_bounds__(E == 64 ? 256 : 512)
+quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
+    extern __shared__ float xsm[];                 // [E][blockDim.x] exchange, then [warps] partial sums
+    constexpr int H = E / 2;                       // float2 pairs per thread
+    pdl_launch_dependents();
+    pdl_wait();
+    const int tid = threadIdx.x;
+    const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
+    const QuantTensor &tn = a.t[which];
+    const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
+    const int S = a.S;
+    const int r_local = tid / S;
+    const int tr = tid - r_local * S;              // slot inside the row
+    const long long row = (long long)blk * a.R + r_local;
+    const int T = a.cols / E;
+    const bool active = (row < tn.rows) && (tr < T);
+
+    float2 v[H];
+    if (active) {
+        if (BF16) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(tn.x) + row * tn.ld + (long long)tr * E);
+#pragma unroll
+            for (int q = 0; q < E / 8; ++q) {
+                const uint4 w = __ldg(src + q);
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    v[q * 4 + j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
+            }
+        } else {
+            const float4 *src = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(tn.x) + row * tn.ld + (long long)tr * E);
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) {
+                const float4 w = __ldg(src + q);
+                v[q * 2] = make_float2(w.x, w.y);
+                v[q * 2 + 1] = make_float2(w.z, w.w);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
+    }
+    rotate_project_store<CB, E, false>(v, a, tn, active, row, tr, r_local, xsm, a.had_block >> 1);
+}
+
+// Streaming variant for bfloat16 rows (E = 64, had_block >= 64): a persistent grid in which every
+// thread prefetches its 128 bytes of the NEXT row group into a private, padded shared-memory slot
+// with cp.async while it works on the current one, so HBM latency hides behind the arithmetic
+// whatever the occupancy.  Slots are 144 bytes apart: the 16-byte reads of a quarter warp fall in
+// distinct bank groups.  Slots past the row end and rows past the tensor end are filled with zeros
+// (source size 0), so reads need no predicate.  The first butterfly stage (stride had_block/2)
+// pairs this thread with thread tid ^ dist0 of the same row; both read both raw slots from shared
+// memory, so that stage needs no shuffles.
+template <int CB, int E>
+__global__ void __launch_bounds__(256, E == 64 ? 2 : 4)
+quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, int exchange_bytes) {
+    constexpr int H = E / 2;
+    constexpr int STREAM_SLOT = 2 * E + 16;
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    pdl_launch_dependents();
+    pdl_wait();
+    float *xsm = reinterpret_cast<float *>(smem_raw);
+    uint8_t *stage = smem_raw + exchange_bytes;
+    const int tid = threadIdx.x;
+    const int nthreads = blockDim.x;
+    const int r_local = tid / a.S;
+    const int tr = tid - r_local * a.S;
+    const bool slot_ok = tr < a.cols / E;
+    const uint32_t my_slot = (uint32_t)__cvta_generic_to_shared(stage) + (uint32_t)tid * STREAM_SLOT;
+    const uint32_t buf_stride = (uint32_t)nthreads * STREAM_SLOT;
+
+    auto locate = [&](int grp, int &which, long long &row) {
+        which = grp >= a.blocks0 ? 1 : 0;
+        row = (long long)(which ? grp - a.blocks0 : grp) * a.R + r_local;
+    };
+    auto prefetch = [&](int grp, int buf) {
+        if (grp < total_groups) {
+            int which;
+            long long row;
+            locate(grp, which, row);
+            const QuantTensor &tn = a.t[which];
+            const bool live = slot_ok && row < tn.rows;
+            const uint8_t *src = live ? reinterpret_cast<const uint8_t *>(tn.x) + (row * tn.ld + (long long)tr * E) * 2
+                                      : reinterpret_cast<const uint8_t *>(tn.x);
+            const uint32_t nbytes = live ? 16u : 0u;
+            const uint32_t step = live ? 16u : 0u;
+            const uint32_t dst = my_slot + (uint32_t)buf * buf_stride;
+#pragma unroll
+            for (int q = 0; q < E / 8; ++q)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + q * 16), "l"(src + q * step),
+                             "r"(nbytes)
+                             : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto widen = [](const uint4 &w, float2 *out) {
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out[j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
+    };
+
+    const bool first_from_smem = a.had_block >= 2 * E;
+    const int dist0 = first_from_smem ? (a.had_block >> 1) / E : 0;
+    const bool cross_warp = dist0 >= 32;
+    const float sg0 = (tid & dist0) ? -1.0f : 1.0f;
+    const float2 sgn0 = make_float2(sg0, sg0);
+    const int s_start = first_from_smem ? (a.had_block >> 2) : (a.had_block >> 1);
+
+    int buf = 0;
+    prefetch((int)blockIdx.x, 0);
+    for (int grp = (int)blockIdx.x; grp < total_groups; grp += (int)gridDim.x, buf ^= 1) {
+        // the slot about to be refilled was read by the partner thread one iteration ago
+        if (cross_warp) __syncthreads(); else __syncwarp();
+        prefetch(grp + (int)gridDim.x, buf ^ 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        if (cross_warp) __syncthreads(); else __syncwarp();   // the partner's copies have landed too
+        int which;
+        long long row;
+        locate(grp, which, row);
+        const QuantTensor &tn = a.t[which];
+        const bool active = slot_ok && row < tn.rows;
+        float2 v[H];
+        const uint8_t *bufp = stage + (size_t)buf * buf_stride;
+        const uint4 *own = reinterpret_cast<const uint4 *>(bufp + (size_t)tid * STREAM_SLOT);
+        if (first_from_smem) {
+            const uint4 *oth = reinterpret_cast<const uint4 *>(bufp + (size_t)(tid ^ dist0) * STREAM_SLOT);
+#pragma unroll
+            for (int q = 0; q < E / 8; ++q) {
+                float2 o[4], p[4];
+                widen(own[q], o);
+                widen(oth[q], p);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[q * 4 + j] = __ffma2_rn(o[j], sgn0, p[j]);   // own * (+-1) + partner
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < E / 8; ++q) widen(own[q], &v[q * 4]);
+        }
+        rotate_project_store<CB, E, true>(v, a, tn, active, row, tr, r_local, xsm, s_start);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 template <bool BF16, int E>
 static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
@@ -400,6 +509,26 @@ static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cuda
     return cudaGetLastError();
 }
 
+template <int E>
+static cudaError_t launch_stream(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                                 int total_groups, int exchange_bytes) {
+#define QUEST_LAUNCH(CBV)                                                                                   \
+    do {                                                                                                    \
+        cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<CBV, E>,                               \
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);     \
+        if (e_ != cudaSuccess) return e_;                                                                   \
+        return launch_pdl(quantize_stream_kernel<CBV, E>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
+                          total_groups, exchange_bytes);                                                    \
+    } while (0)
+    switch (cb) {
+        case 1: QUEST_LAUNCH(1);
+        case 2: QUEST_LAUNCH(2);
+        case 4: QUEST_LAUNCH(4);
+        default: QUEST_LAUNCH(8);
+    }
+#undef QUEST_LAUNCH
+}
+
 }  // namespace
 
 int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
@@ -407,7 +536,10 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
     const QuantConsts qc = make_quant_consts(bits, had_block, trust_factor);
     const int cb = container_bits(bits);
     if (cols % 32 == 0) {
-        const int E = (cols % 64 == 0) ? 64 : 32;
+        // streaming kernel with 32 elements per thread (64 registers, twice the resident warps) measured
+        // faster than 64 per thread for rows up to 4096 elements; wider rows keep 64 per thread
+        const bool stream32 = dtype == QUEST_BF16 && had_block >= 64 && cols <= 4096;
+        const int E = (cols % 64 == 0 && !stream32) ? 64 : 32;
         const int T = (int)(cols / E);
         int S;
         if (T < 32) { S = 1; while (S < T) S <<= 1; } else { S = (T + 31) / 32 * 32; }
@@ -436,7 +568,19 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = S; a.R = R;
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
-            if (E == 64)
+            if ((E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64) {
+                // persistent streaming kernel: as many CTAs as fit on the device, each looping over groups
+                const int exchange = (int)((smem + 15) / 16 * 16);
+                const size_t smem2 = (size_t)exchange + 2 * (size_t)threads * (2 * E + 16);
+                int dev = 0, sms = 148;
+                cudaGetDevice(&dev);
+                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+                const int per_sm = smem2 > 100 * 1024 ? 1 : (E == 64 ? 2 : 4);
+                const int total = nb[0] + nb[1];
+                const int g = total < sms * per_sm ? total : sms * per_sm;
+                e = E == 64 ? launch_stream<64>(cb, g, threads, smem2, st, a, total, exchange)
+                            : launch_stream<32>(cb, g, threads, smem2, st, a, total, exchange);
+            } else if (E == 64)
                 e = dtype == QUEST_BF16 ? launch_rows<true, 64>(cb, grid, threads, smem, st, a)
                                         : launch_rows<false, 64>(cb, grid, threads, smem, st, a);
             else
