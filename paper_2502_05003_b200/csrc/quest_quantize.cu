@@ -158,8 +158,10 @@ struct QuantArgs {
 
 // Everything after the load: rotation from stride s_start downwards (larger strides already
 // applied by the caller), RMS, projection, trust test, packing and stores for the E elements this
-// thread holds.  GFULL: had_block >= E, so every in-register stage runs.
-template <int CB, int E, bool GFULL>
+// thread holds.  GFULL: had_block >= E, so every in-register stage runs.  FAST: the common case
+// fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
+// one warp, every output requested, no row sums -- so that no per-row branch or loop remains.
+template <int CB, int E, bool GFULL, bool FAST>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
                                                      int s_start) {
@@ -172,7 +174,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
     const int had_block = a.had_block;
     // ---- rotation, descending stride --------------------------------------------------------
     const float2 neg1 = make_float2(-1.0f, -1.0f);
-    for (int s = s_start; s >= 32 * E; s >>= 1) {             // partner thread is in another warp
+    for (int s = FAST ? 0 : s_start; s >= 32 * E; s >>= 1) {  // partner thread is in another warp
         const int dist = s / E;
         float2 *x2 = reinterpret_cast<float2 *>(xsm);
         __syncthreads();
@@ -185,7 +187,19 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
 #pragma unroll
         for (int i = 0; i < H; ++i) v[i] = __ffma2_rn(v[i], sgn, x2[i * nthreads + pt]);
     }
-    {
+    if constexpr (FAST) {
+        if constexpr (E == 32) {                               // stride 32: partner is the neighbouring lane
+            const float sg = (lane & 1) ? -1.0f : 1.0f;
+            const float2 sgn = make_float2(sg, sg);
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+                float2 p;
+                p.x = __shfl_xor_sync(0xffffffffu, v[i].x, 1);
+                p.y = __shfl_xor_sync(0xffffffffu, v[i].y, 1);
+                v[i] = __ffma2_rn(v[i], sgn, p);
+            }
+        }
+    } else {
         int s0 = s_start;
         if (s0 > 16 * E) s0 = 16 * E;
 #pragma unroll 1
@@ -238,8 +252,13 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
             for (int i = 0; i < n; ++i) q[i] = __fadd_rn(q[2 * i], q[2 * i + 1]);
         ss = q[0];
     }
-    const int lanes_per_row = S < 32 ? S : 32;
-    for (int m = 1; m < lanes_per_row; m <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, m));
+    const int lanes_per_row = (FAST || S >= 32) ? 32 : S;
+    if constexpr (FAST) {
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, m));
+    } else {
+        for (int m = 1; m < lanes_per_row; m <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, m));
+    }
     if (S > 32) {
         const int nw = S >> 5;                                  // warps per row
         int nwp2 = 1;
@@ -254,7 +273,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
     }
     const float rms = __fsqrt_rn(__fdiv_rn(ss, (float)cols));
     const float inv = (rms > 0.0f) ? __fdiv_rn(a.qc.A, rms) : 0.0f;
-    if (active && tn.scales && tr == 0) tn.scales[row] = __fmul_rn(rms, a.qc.B);
+    if (active && (FAST || tn.scales) && tr == 0) tn.scales[row] = __fmul_rn(rms, a.qc.B);
 
     // ---- project: level axis, clamp, round to nearest even, trust test -----------------------
     const float2 inv2 = make_float2(inv, inv), c02 = make_float2(a.qc.c0, a.qc.c0);
@@ -284,7 +303,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 kb[2 * i + 1] = __float_as_uint(km.y);
             }
             mbits = ~mbits;
-            if (tn.mask)
+            if (FAST || tn.mask)
                 reinterpret_cast<uint32_t *>(tn.mask + row * (long long)(cols >> 3))[tr * (E / 32) + g32] = mbits;
 
             // pack 32/CB codes per word: sum_j (MAGIC_BITS + k_j) * 2^(CB*j), minus the constant part
@@ -300,7 +319,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 for (int j = PER - 1; j >= 0; --j) acc = (acc << CB) + kb[q * PER + j];
                 w[q] = acc - magic_sum;
             }
-            if (tn.codes) {
+            if (FAST || tn.codes) {
                 uint8_t *dst = tn.codes + row * (long long)(cols * CB / 8) + ((long long)tr * (E / 32) + g32) * (4 * CB);
                 if constexpr (CB == 8) {
                     reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -313,20 +332,20 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                     reinterpret_cast<uint32_t *>(dst)[0] = w[0];
                 }
             }
-            if (tn.op8) {
+            if (FAST || tn.op8) {
                 uint32_t o[8];
                 operand_from_code_words<CB>(w, a.bits, o);
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                if (tn.rowsum) {
+                if (!FAST && tn.rowsum) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q) rsum += sum_bytes_s8(o[q]);
                 }
             }
         }
     }
-    if (tn.rowsum) {                                            // uniform over the CTA
+    if (!FAST && tn.rowsum) {                                   // uniform over the CTA
         for (int m = 1; m < lanes_per_row; m <<= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, m);
         if (S > 32) {
             int *ism = reinterpret_cast<int *>(xsm);
@@ -386,7 +405,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
 #pragma unroll
         for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
     }
-    rotate_project_store<CB, E, false>(v, a, tn, active, row, tr, r_local, xsm, a.had_block >> 1);
+    rotate_project_store<CB, E, false, false>(v, a, tn, active, row, tr, r_local, xsm, a.had_block >> 1);
 }
 
 // Streaming variant for bfloat16 rows (E = 64, had_block >= 64): a persistent grid in which every
@@ -397,7 +416,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
 // (source size 0), so reads need no predicate.  The first butterfly stage (stride had_block/2)
 // pairs this thread with thread tid ^ dist0 of the same row; both read both raw slots from shared
 // memory, so that stage needs no shuffles.
-template <int CB, int E>
+template <int CB, int E, bool FAST>
 __global__ void __launch_bounds__(256, E == 64 ? 2 : 4)
 quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, int exchange_bytes) {
     constexpr int H = E / 2;
@@ -445,12 +464,12 @@ quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, in
         for (int j = 0; j < 4; ++j) out[j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
     };
 
-    const bool first_from_smem = a.had_block >= 2 * E;
-    const int dist0 = first_from_smem ? (a.had_block >> 1) / E : 0;
-    const bool cross_warp = dist0 >= 32;
+    const bool first_from_smem = FAST || a.had_block >= 2 * E;
+    const int dist0 = FAST ? 64 / E : first_from_smem ? (a.had_block >> 1) / E : 0;
+    const bool cross_warp = !FAST && dist0 >= 32;
     const float sg0 = (tid & dist0) ? -1.0f : 1.0f;
     const float2 sgn0 = make_float2(sg0, sg0);
-    const int s_start = first_from_smem ? (a.had_block >> 2) : (a.had_block >> 1);
+    const int s_start = FAST ? 32 : first_from_smem ? (a.had_block >> 2) : (a.had_block >> 1);
 
     int buf = 0;
     prefetch((int)blockIdx.x, 0);
@@ -482,7 +501,7 @@ quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, in
 #pragma unroll
             for (int q = 0; q < E / 8; ++q) widen(own[q], &v[q * 4]);
         }
-        rotate_project_store<CB, E, true>(v, a, tn, active, row, tr, r_local, xsm, s_start);
+        rotate_project_store<CB, E, true, FAST>(v, a, tn, active, row, tr, r_local, xsm, s_start);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -509,15 +528,15 @@ static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cuda
     return cudaGetLastError();
 }
 
-template <int E>
+template <int E, bool FAST>
 static cudaError_t launch_stream(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                  int total_groups, int exchange_bytes) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
-        cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<CBV, E>,                               \
+        cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<CBV, E, FAST>,                               \
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);     \
         if (e_ != cudaSuccess) return e_;                                                                   \
-        return launch_pdl(quantize_stream_kernel<CBV, E>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
+        return launch_pdl(quantize_stream_kernel<CBV, E, FAST>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
                           total_groups, exchange_bytes);                                                    \
     } while (0)
     switch (cb) {
@@ -578,8 +597,17 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 const int per_sm = smem2 > 100 * 1024 ? 1 : (E == 64 ? 2 : 4);
                 const int total = nb[0] + nb[1];
                 const int g = total < sms * per_sm ? total : sms * per_sm;
-                e = E == 64 ? launch_stream<64>(cb, g, threads, smem2, st, a, total, exchange)
-                            : launch_stream<32>(cb, g, threads, smem2, st, a, total, exchange);
+                bool fast = had_block == 128 && S >= 32 && bits < 8;
+                for (int j = 0; j < 2; ++j) {
+                    const QuantTensor &t = a.t[j];
+                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum)) fast = false;
+                }
+                if (fast)
+                    e = E == 64 ? launch_stream<64, true>(cb, g, threads, smem2, st, a, total, exchange)
+                                : launch_stream<32, true>(cb, g, threads, smem2, st, a, total, exchange);
+                else
+                    e = E == 64 ? launch_stream<64, false>(cb, g, threads, smem2, st, a, total, exchange)
+                                : launch_stream<32, false>(cb, g, threads, smem2, st, a, total, exchange);
             } else if (E == 64)
                 e = dtype == QUEST_BF16 ? launch_rows<true, 64>(cb, grid, threads, smem, st, a)
                                         : launch_rows<false, 64>(cb, grid, threads, smem, st, a);
