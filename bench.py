@@ -37,8 +37,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, taken from the
 # committed ncu summary (profiles/); None until a capture exists.
-GEMM_DRAM_TRAFFIC_BYTES = None
-QUANT_DRAM_TRAFFIC_BYTES = None
+GEMM_DRAM_TRAFFIC_BYTES = 12651008          # profiles/gemm_i8_config2_full.md
+QUANT_DRAM_TRAFFIC_BYTES = 25188096         # profiles/quantize_stream_config2_full.md (x and w in one launch)
+QUANT_INSTR_PER_ELEMENT = 24.9              # thread instructions per element, same profile
 
 
 def load_peaks():
@@ -410,7 +411,16 @@ def run_gpu(args, rank: int, world: int, local: int):
         "roofline_quantizer": {"bound": "hbm", "kernel": "quantizer, x and w rows in one launch", "achieved": q_gbs,
                                "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": (q_gbs / peaks["hbm_gbs"]) if q_gbs else None, "peak_basis": src,
-                               "traffic": QUANT_DRAM_TRAFFIC_BYTES, "ms": q_ms, "algorithmic_bytes": q_bytes},
+                               "traffic": QUANT_DRAM_TRAFFIC_BYTES, "ms": q_ms, "algorithmic_bytes": q_bytes,
+                               # the kernel is bound by instruction issue, not HBM: the same launch against the
+                               # issue rate 148 SMs x 4 schedulers x 32 lanes x SM clock
+                               "alu": (lambda mhz: {"bound": "alu", "unit": "T thread-instr/s",
+                                                    "achieved": QUANT_INSTR_PER_ELEMENT * (M + N) * K / (q_ms * 1e-3) / 1e12,
+                                                    "peak": 148 * 4 * 32 * mhz * 1e6 / 1e12,
+                                                    "frac": QUANT_INSTR_PER_ELEMENT * (M + N) * K / (q_ms * 1e-3)
+                                                            / (148 * 4 * 32 * mhz * 1e6),
+                                                    "instr_per_element": QUANT_INSTR_PER_ELEMENT})(
+                                   clocks.summary()["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)) if q_ms else None},
         "stage_ms": stage_ms,
         "cpu_baseline": {"value": sample / o_dt, "unit": UNIT, "cores": o_threads, "kind": "oracle",
                          "sample": f"{sample} of {TOKENS} token rows against the full W, one pass"},
