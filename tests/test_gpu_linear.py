@@ -85,3 +85,36 @@ def test_config5_points(bits, d, tokens):
     rows = np.random.default_rng(3).choice(tokens, 32, replace=False)
     for g in (128, d):
         check_linear(p["x"], p["w"], bits, g, 1.0, torch.bfloat16, BF16_OUT_RTOL, sample_rows=rows)
+
+
+def test_linear_fwd_replays_from_a_cuda_graph():
+    """Section 5 runs the whole pipeline under a CUDA graph: the call must be capturable (no
+    allocation, no synchronisation) and every replay must reproduce the directly launched result."""
+    import paper_2502_05003_b200 as quest
+    c = synth.config2(tokens=512)
+    x, w = to_dev(c["x"]), to_dev(c["w"])
+    ref = quest.quest_linear_fwd(x, w, 4, 128, 1.0, out_dtype=torch.bfloat16)
+    M, K = x.shape
+    N = w.shape[0]
+    saved = {"xq": torch.zeros_like(ref["xq"]), "sx": torch.zeros_like(ref["sx"]), "mx": torch.zeros_like(ref["mx"]),
+             "wq": torch.zeros_like(ref["wq"]), "sw": torch.zeros_like(ref["sw"]), "mw": torch.zeros_like(ref["mw"])}
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = quest.alloc_workspace(M, N, K, 4, 4)
+    torch.cuda.synchronize()
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        quest.quest_linear_fwd(x, w, 4, 128, 1.0, y=y, saved=saved, workspace=ws)     # warm-up outside the capture
+        st.synchronize()
+        with torch.cuda.graph(g, stream=st):
+            quest.quest_linear_fwd(x, w, 4, 128, 1.0, y=y, saved=saved, workspace=ws)
+    for _ in range(3):
+        y.zero_()
+        for t in saved.values():
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(y, ref["y"])
+        for k in saved:
+            assert torch.equal(saved[k], ref[k]), k
+    assert quest.quest_device_status() == 0
