@@ -162,6 +162,36 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
                      uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * quest_linear_bwd -- Algorithm 2 (QuEST training backward) for one linear layer, from what
+ * quest_linear_fwd saved:
+ *
+ *     dL/dxq_h = dL/dy wq_h;   dL/dx = IHT(M(x_h; xq_h) * dL/dxq_h)
+ *     dL/dwq_h = dL/dy^T xq_h; dL/dw = IHT(M(w_h; wq_h) * dL/dwq_h)
+ *
+ * with the trust estimator of Section 3.2 applied in the Hadamard domain and IHT the inverse of
+ * the orthonormal block Hadamard transform.  The two products run on the tensor cores with
+ * bfloat16 operands and binary32 accumulation ("standard 16-bit precision", Section 3.3): the grid
+ * values are exact in bfloat16 and the per-row scale of the quantized operand is folded into dL/dy
+ * before it is rounded to bfloat16.
+ *
+ *   dy                 device, [M x N] bfloat16, dense, 16-byte aligned
+ *   M, N, K            M, N > 0 and multiples of 8; 32 <= K <= 16384, K % 32 == 0
+ *   bits, had_block    as in the forward call that produced the codes
+ *   xq, sx, mx         device: codes [M x K], scales [M], trust mask [M x K/8] of x (forward outputs)
+ *   wq, sw, mw         the same for w ([N x K])
+ *   dx, dw             device out: [M x K] and [N x K], dense, out_dtype (QUEST_F32 or QUEST_BF16),
+ *                      16-byte aligned; either may be NULL to skip that gradient
+ *   workspace          device scratch of at least quest_bwd_workspace_bytes(M, N, K) bytes, 256-byte
+ *                      aligned (bfloat16 operands and the masked binary32 products)
+ */
+int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K, int bits, int had_block,
+                     const uint8_t *xq, const float *sx, const uint8_t *mx,
+                     const uint8_t *wq, const float *sw, const uint8_t *mw,
+                     void *dx, void *dw, int out_dtype,
+                     void *workspace, size_t workspace_bytes, void *stream);
+size_t quest_bwd_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
 /* Bytes of scratch quest_lowbit_gemm / quest_linear_fwd need (0 on invalid arguments). */
 size_t quest_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w);
 

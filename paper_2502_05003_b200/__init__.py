@@ -204,3 +204,34 @@ def quest_linear_fwd(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int
     _lib.check(st)
     out["y"] = y
     return out
+
+
+def quest_bwd_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(_lib.load().quest_bwd_workspace_bytes(M, N, K))
+
+
+def quest_linear_bwd(dy: torch.Tensor, fwd: dict, bits: int, had_block: int, K: int, out_dtype=torch.float32,
+                     dx: torch.Tensor = None, dw: torch.Tensor = None, want_dx: bool = True, want_dw: bool = True,
+                     workspace: torch.Tensor = None) -> dict:
+    """Algorithm 2 from the forward call's saved tensors (``fwd`` holds xq, sx, mx, wq, sw, mw).
+    ``dy`` [M, N] bfloat16.  Returns {"dx": [M, K] or None, "dw": [N, K] or None}."""
+    _require_cuda(dy, dx, dw, workspace, *[fwd[k] for k in ("xq", "sx", "mx", "wq", "sw", "mw")])
+    if dy.dtype != torch.bfloat16 or not dy.is_contiguous():
+        raise ValueError("quest_linear_bwd: dy must be a contiguous bfloat16 tensor")
+    M, N = dy.shape
+    if dx is None and want_dx:
+        dx = torch.empty((M, K), dtype=out_dtype, device=dy.device)
+    if dw is None and want_dw:
+        dw = torch.empty((N, K), dtype=out_dtype, device=dy.device)
+    if workspace is None:
+        n = quest_bwd_workspace_bytes(M, N, K)
+        if n == 0:
+            raise ValueError("quest_linear_bwd: unsupported shape (M, N multiples of 8; K a multiple of 32, <= 16384)")
+        workspace = torch.empty(n, dtype=torch.uint8, device=dy.device)
+    out_t = dx if dx is not None else dw
+    st = _lib.load().quest_linear_bwd(_p(dy), M, N, K, bits, had_block, _p(fwd["xq"]), _p(fwd["sx"]), _p(fwd["mx"]),
+                                      _p(fwd["wq"]), _p(fwd["sw"]), _p(fwd["mw"]), _p(dx), _p(dw),
+                                      _dtype_code(out_t) if out_t is not None else 0,
+                                      _p(workspace), workspace.numel(), _stream())
+    _lib.check(st)
+    return {"dx": dx, "dw": dw}

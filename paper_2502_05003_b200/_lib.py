@@ -11,7 +11,7 @@ EXPORTS = (
     "quest_quantize", "quest_trust_mask", "quest_lowbit_gemm", "quest_linear_fwd",
     "quest_workspace_bytes", "quest_codes_bytes", "quest_alpha_star", "quest_device_status",
     "quest_status_string", "quest_last_cuda_error", "quest_stage_timing", "quest_stage_times",
-    "quest_lowbit_gemm_static",
+    "quest_lowbit_gemm_static", "quest_linear_bwd", "quest_bwd_workspace_bytes",
 )
 
 _lib = None
@@ -42,6 +42,10 @@ def load() -> ctypes.CDLL:
     L.quest_lowbit_gemm.argtypes = [vp, vp, ci, vp, vp, ci, i64, i64, i64, vp, ci, i64, vp, vp, sz, vp]
     L.quest_lowbit_gemm_static.restype = ci
     L.quest_lowbit_gemm_static.argtypes = [vp, vp, ci, vp, vp, ci, i64, i64, i64, vp, ci, i64, vp, vp]
+    L.quest_linear_bwd.restype = ci
+    L.quest_linear_bwd.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
+    L.quest_bwd_workspace_bytes.restype = sz
+    L.quest_bwd_workspace_bytes.argtypes = [i64, i64, i64]
     L.quest_linear_fwd.restype = ci
     L.quest_linear_fwd.argtypes = [vp, vp, ci, i64, i64, i64, ci, ci, cf, vp, ci,
                                    vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]

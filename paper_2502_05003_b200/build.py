@@ -22,6 +22,7 @@ UNITS = {
     "quest_quantize.cu": ["-fmad=false"],
     "quest_gemm.cu": [],
     "quest_static.cu": [],
+    "quest_backward.cu": [],
 }
 
 

@@ -50,7 +50,7 @@ constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s at 2 GHz
 enum { ST_OK = 0, ST_PRODUCER = 1, ST_MMA = 2, ST_EPILOGUE = 3 };
 
 struct GemmParams {
-    int M, N, K;
+    int M, N, K;           // K: bytes of the contraction per operand row (int8: elements; bf16: 2 x elements)
     const float *sx;
     const float *sw;
     const int32_t *rs_a;   // row sums of the A operand values (nullable)
@@ -61,6 +61,7 @@ struct GemmParams {
     int y_dtype;
     long long ldy;
     int32_t *acc;
+    const uint8_t *mask;   // backward mode: trust-mask bitmap of the output, [M x N/8] bytes (1 = keep)
     int *status;
 };
 
@@ -136,6 +137,19 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// kind::f16 with bfloat16 operands (both K-major) and binary32 accumulation
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                  : "memory");
@@ -171,6 +185,15 @@ __device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, u
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -220,11 +243,16 @@ struct SmemLayout {
 
 // YT: y leaves through shared memory and TMA tile stores (whole 128-byte row segments per
 // transaction) instead of per-thread 16-byte stores, which write every 32-byte sector twice.
-template <int BN, bool CORR, bool TWO, bool YT>
+// MODE 0: int8 operands, scaled output.  MODE 1: int8 operands with the exact correction for 8-bit
+// codes.  MODE 2 (backward pass, Algorithm 2): bfloat16 operands (kind::f16, binary32 accumulators);
+// the epilogue zeroes the elements the trust mask rejects and stores binary32.
+template <int BN, int MODE, bool TWO, bool YT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
     using L = SmemLayout<BN, TWO>;
+    constexpr bool CORR = MODE == 1;
+    constexpr bool BWD = MODE == 2;
     constexpr int STAGES = L::NSTAGES;
     constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
     extern __shared__ uint8_t smem_raw[];
@@ -326,7 +354,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0 && leader) {
-            constexpr uint32_t idesc = make_idesc_i8(TILE_M, BN);
+            constexpr uint32_t idesc = BWD ? make_idesc_bf16(TILE_M, BN) : make_idesc_i8(TILE_M, BN);
             int stage = 0;
             uint32_t phase = 0;
             int t = 0;
@@ -348,12 +376,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int kk = 0; kk < BK / UMMA_K; ++kk) {
                         // advance along K inside the 128-byte swizzle row: +32 bytes = +2 in 16-byte units
-                        if constexpr (TWO)
-                            umma_i8_pair(d_tmem, a_desc + (uint64_t)(kk * (UMMA_K >> 4)),
-                                         b_desc + (uint64_t)(kk * (UMMA_K >> 4)), idesc, (kb | kk) != 0 ? 1u : 0u);
-                        else
-                            umma_i8(d_tmem, a_desc + (uint64_t)(kk * (UMMA_K >> 4)),
-                                    b_desc + (uint64_t)(kk * (UMMA_K >> 4)), idesc, (kb | kk) != 0 ? 1u : 0u);
+                        const uint64_t ad = a_desc + (uint64_t)(kk * (UMMA_K >> 4));
+                        const uint64_t bd = b_desc + (uint64_t)(kk * (UMMA_K >> 4));
+                        const uint32_t accum = (kb | kk) != 0 ? 1u : 0u;
+                        if constexpr (BWD) {      // 32 bytes of K = 16 bfloat16 per instruction
+                            if constexpr (TWO) umma_bf16_pair(d_tmem, ad, bd, idesc, accum);
+                            else umma_bf16(d_tmem, ad, bd, idesc, accum);
+                        } else {
+                            if constexpr (TWO) umma_i8_pair(d_tmem, ad, bd, idesc, accum);
+                            else umma_i8(d_tmem, ad, bd, idesc, accum);
+                        }
                     }
                     // stage reusable (in both CTAs of a pair) once these MMAs retire
                     if constexpr (TWO) umma_commit_pair(smem_u32(&empty_bar[stage]));
@@ -393,7 +425,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int32_t *cbt = cb_tile + buf * BN;
             for (int c = ep_tid; c < BN; c += 32 * EPI_WARPS) {
                 const int col = n0 + c;
-                swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
+                if (!BWD) swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
                 if (CORR) cbt[c] = (p.rs_b && col < p.N) ? p.cb * __ldg(p.rs_b + col) : 0;
             }
             const int row = m0 + quarter * 32 + lane;
@@ -401,7 +433,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // without 8-bit corrections and without the raw accumulators, the exact power of two of the
             // operand scaling is folded into the row scale instead of shifting every accumulator
             const bool fold = !CORR && !p.acc;
-            float sxr = (row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
+            float sxr = (!BWD && row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
             if (fold) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.sh) << 23));
             int rsa = 0;
             if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
@@ -444,7 +476,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (col0 < p.N) {                      // uniform across the warp
                     const bool full = col0 + 32 <= p.N;
                     uint32_t *rc = &r[c0];
-                    if (CORR) {
+                    if constexpr (BWD) {
+                        // trust estimator: keep the gradient only where the forward mask trusts the element
+                        const uint32_t mbits = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(
+                                                            p.mask + (long long)row * (p.N >> 3) + (col0 >> 3)))
+                                                      : 0u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) rc[j] = ((mbits >> j) & 1u) ? rc[j] : 0u;
+                    } else if (CORR) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
                             rc[j] = (uint32_t)((int32_t)((uint32_t)p.mul * rc[j] + (uint32_t)rsa +
@@ -453,7 +492,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 32; ++j) rc[j] = (uint32_t)((int32_t)rc[j] >> p.sh);
                     }
-                    if (p.acc && row_ok) {
+                    if (!BWD && p.acc && row_ok) {
                         int32_t *dst = p.acc + (long long)row * p.N + col0;
                         if (vec_acc && full) {
 #pragma unroll
@@ -470,7 +509,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const float2 sx2 = make_float2(sxr, sxr);
                         const float2 *sw2 = reinterpret_cast<const float2 *>(swt + cbase + c0);
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
+                        for (int j = 0; j < (BWD ? 0 : 32); j += 2) {
                             const float2 a2 = make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
                             const float2 y2 = __fmul2_rn(__fmul2_rn(sx2, sw2[j >> 1]), a2);
                             rc[j] = __float_as_uint(y2.x);
@@ -670,13 +709,13 @@ int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes
     return QUEST_OK;
 }
 
-template <int BN, bool CORR, bool TWO, bool YT>
+template <int BN, int MODE, bool TWO, bool YT>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
                    cudaStream_t st) {
     using L = SmemLayout<BN, TWO>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, CORR, TWO, YT>,
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, MODE, TWO, YT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
         attr_done = true;
@@ -693,7 +732,7 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
     } else {
         grid = tiles < sms ? tiles : sms;
     }
-    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, CORR, TWO, YT>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
+    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
                                TWO ? 2 : 1, tmA, tmB, tmY, p);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
@@ -758,7 +797,7 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
     else { p.mul = 2; p.ca = 1; p.cb = 0; p.ck = 0; p.sh = 7 - bits_x; }
     p.rs_a = p.ca ? rs_a : nullptr;                      // row sums of the x operand bytes
     p.rs_b = p.cb ? rs_b : nullptr;                      // row sums of the w operand bytes
-    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
 
@@ -779,14 +818,40 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
         if (s) return s;
     }
 #define QUEST_GEMM(BNV, TWOV)                                                                        \
-    (corr ? (yt ? launch_gemm_bn<BNV, true, TWOV, true>(tmA, tmB, tmY, p, st)                         \
-                : launch_gemm_bn<BNV, true, TWOV, false>(tmA, tmB, tmY, p, st))                        \
-          : (yt ? launch_gemm_bn<BNV, false, TWOV, true>(tmA, tmB, tmY, p, st)                        \
-                : launch_gemm_bn<BNV, false, TWOV, false>(tmA, tmB, tmY, p, st)))
+    (corr ? (yt ? launch_gemm_bn<BNV, 1, TWOV, true>(tmA, tmB, tmY, p, st)                            \
+                : launch_gemm_bn<BNV, 1, TWOV, false>(tmA, tmB, tmY, p, st))                           \
+          : (yt ? launch_gemm_bn<BNV, 0, TWOV, true>(tmA, tmB, tmY, p, st)                            \
+                : launch_gemm_bn<BNV, 0, TWOV, false>(tmA, tmB, tmY, p, st)))
     if (pair) return QUEST_GEMM(256, true);
     if (wide) return QUEST_GEMM(256, false);
     return QUEST_GEMM(128, false);
 #undef QUEST_GEMM
+}
+
+// Backward-pass contraction (Algorithm 2, lines 2 and 4): out[i][j] = mask[i][j] * sum_k a[i][k] b[j][k]
+// with bfloat16 operands a [I x Kc], b [J x Kc] (both dense, Kc contiguous) and binary32 output [I x J].
+int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
+                            const uint8_t *mask, float *out, cudaStream_t st) {
+    if (I == 0 || J == 0) return QUEST_OK;
+    GemmParams p;
+    p.M = (int)I; p.N = (int)J; p.K = (int)(2 * Kc);
+    p.sx = nullptr; p.sw = nullptr; p.rs_a = nullptr; p.rs_b = nullptr;
+    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
+    p.y = out; p.y_dtype = QUEST_F32; p.ldy = J; p.acc = nullptr; p.mask = mask;
+    p.status = device_status_word();
+    if (!p.status) return QUEST_ERR_CUDA;
+    const bool wide = J > 128;
+    const bool pair = wide && I > 128;
+    CUtensorMap tmA, tmB, tmY;
+    int s = make_operand_map(&tmA, reinterpret_cast<const int8_t *>(a), I, 2 * Kc, BM);
+    if (s) return s;
+    s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(b), J, 2 * Kc, pair ? 128 : wide ? 256 : 128);
+    if (s) return s;
+    s = make_output_map(&tmY, out, I, J * 4, J * 4);
+    if (s) return s;
+    if (pair) return launch_gemm_bn<256, 2, true, true>(tmA, tmB, tmY, p, st);
+    if (wide) return launch_gemm_bn<256, 2, false, true>(tmA, tmB, tmY, p, st);
+    return launch_gemm_bn<128, 2, false, true>(tmA, tmB, tmY, p, st);
 }
 
 }  // namespace quest

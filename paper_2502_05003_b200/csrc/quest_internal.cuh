@@ -116,4 +116,7 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
                 int32_t *acc, cudaStream_t st);
 
+int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
+                            const uint8_t *mask, float *out, cudaStream_t st);
+
 }  // namespace quest

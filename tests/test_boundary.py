@@ -125,3 +125,19 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(_lib, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         _lib.load()
+
+
+def test_backward_argument_errors(lib):
+    def call(**kw):
+        a = dict(dy=FAKE, M=64, N=64, K=128, bits=4, g=128, xq=FAKE, sx=FAKE, mx=FAKE, wq=FAKE, sw=FAKE, mw=FAKE,
+                 dx=FAKE, dw=FAKE, out=0, ws=FAKE, ws_bytes=1 << 30)
+        a.update(kw)
+        return lib.quest_linear_bwd(a["dy"], a["M"], a["N"], a["K"], a["bits"], a["g"], a["xq"], a["sx"], a["mx"],
+                                    a["wq"], a["sw"], a["mw"], a["dx"], a["dw"], a["out"], a["ws"], a["ws_bytes"], None)
+    assert call(dy=None) == 1 and call(mx=None) == 1 and call(dx=None, dw=None) == 1
+    assert call(bits=9) == 3 and call(M=60) == 2 and call(N=0) == 2 and call(K=48) == 2 and call(K=32768) == 2
+    assert call(g=96) == 4 and call(g=256) == 4 and call(out=7) == 5
+    assert call(dy=ctypes.c_void_p(0x10002)) == 6 and call(ws_bytes=16) == 8 and call(ws=None) == 8
+    assert lib.quest_bwd_workspace_bytes(4096, 2048, 2048) >= (2 * 4096 * 2048 + 2048 * 2048 + 4096 * 2048) * 2 + \
+        (4096 + 2048) * 2048 * 4
+    assert lib.quest_bwd_workspace_bytes(60, 64, 128) == 0
