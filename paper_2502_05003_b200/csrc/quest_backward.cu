@@ -12,6 +12,8 @@
 //   2. codes_to_bf16_t_kernel ct[k][r] = bf16(c[r][k])  for w and x   (K-major operands)
 //   3. gemm (quest_gemm.cu, bfloat16 mode): masked binary32 products  d1 [M x K], d2 [N x K]
 //   4. iht_rows_kernel        block Hadamard transform, 1/sqrt(g), store in the output type
+//      (for blocks of 128 stages 3 and 4 are one kernel: the transform runs in the GEMM epilogue,
+//      where a thread holds exactly one block of its output row)
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -249,16 +251,25 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
                        (int)N, (int)K, ws.cwt);
         if (e != cudaSuccess) return cuda_fail(e);
         // line 2 and the mask of line 3: d1[m][k] = M_x[m][k] * sum_n a1[m][n] cwt[k][n]
-        if ((s = launch_gemm_bf16_masked(ws.a1, ws.cwt, M, K, N, mx, ws.d1, st))) return s;
-        if ((s = launch_iht(ws.d1, M, K, had_block, dx, out_dtype, K, st))) return s;
+        // (blocks of 128: the inverse transform is fused into the contraction's epilogue)
+        if (had_block == 128 && M > 128 && K > 128) {
+            if ((s = launch_gemm_bf16_masked(ws.a1, ws.cwt, M, K, N, mx, dx, out_dtype, true, st))) return s;
+        } else {
+            if ((s = launch_gemm_bf16_masked(ws.a1, ws.cwt, M, K, N, mx, ws.d1, QUEST_F32, false, st))) return s;
+            if ((s = launch_iht(ws.d1, M, K, had_block, dx, out_dtype, K, st))) return s;
+        }
     }
     if (dw) {
         e = launch_pdl(codes_to_bf16_t_kernel, dim3((unsigned)((K + 31) / 32), (unsigned)((M + 31) / 32)), blk, 0, st, 1, xq, bits,
                        (int)M, (int)K, ws.cxt);
         if (e != cudaSuccess) return cuda_fail(e);
         // line 4 and the mask of line 5: d2[n][k] = M_w[n][k] * sum_m a2[n][m] cxt[k][m]
-        if ((s = launch_gemm_bf16_masked(ws.a2, ws.cxt, N, K, M, mw, ws.d2, st))) return s;
-        if ((s = launch_iht(ws.d2, N, K, had_block, dw, out_dtype, K, st))) return s;
+        if (had_block == 128 && N > 128 && K > 128) {
+            if ((s = launch_gemm_bf16_masked(ws.a2, ws.cxt, N, K, M, mw, dw, out_dtype, true, st))) return s;
+        } else {
+            if ((s = launch_gemm_bf16_masked(ws.a2, ws.cxt, N, K, M, mw, ws.d2, QUEST_F32, false, st))) return s;
+            if ((s = launch_iht(ws.d2, N, K, had_block, dw, out_dtype, K, st))) return s;
+        }
     }
     return QUEST_OK;
 }

@@ -245,14 +245,18 @@ struct SmemLayout {
 // transaction) instead of per-thread 16-byte stores, which write every 32-byte sector twice.
 // MODE 0: int8 operands, scaled output.  MODE 1: int8 operands with the exact correction for 8-bit
 // codes.  MODE 2 (backward pass, Algorithm 2): bfloat16 operands (kind::f16, binary32 accumulators);
-// the epilogue zeroes the elements the trust mask rejects and stores binary32.
+// the epilogue zeroes the elements the trust mask rejects and stores binary32.  MODE 3: MODE 2 plus
+// the inverse Hadamard transform for blocks of 128 fused into the epilogue (BN = 256: the 128
+// columns a thread holds are exactly one block), output in the caller's type.
 template <int BN, int MODE, bool TWO, bool YT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
     using L = SmemLayout<BN, TWO>;
     constexpr bool CORR = MODE == 1;
-    constexpr bool BWD = MODE == 2;
+    constexpr bool BWD = MODE >= 2;
+    constexpr bool IHT128 = MODE == 3;
+    static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
     constexpr int STAGES = L::NSTAGES;
     constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
     extern __shared__ uint8_t smem_raw[];
@@ -470,13 +474,47 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if constexpr (TWO) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[buf]), 0));   // the leader's barrier
                 else mbar_arrive(smem_u32(&tempty_bar[buf]));
             }
+            if constexpr (IHT128) {
+                // lines 3 / 5 of Algorithm 2 on this thread's block of 128: mask, then the inverse
+                // orthonormal Hadamard transform in registers (descending stride, packed binary32)
+                if (n0 + cbase < p.N) {
+                    uint4 mb = make_uint4(0u, 0u, 0u, 0u);
+                    if (row_ok) mb = __ldg(reinterpret_cast<const uint4 *>(p.mask + (long long)row * (p.N >> 3) + ((n0 + cbase) >> 3)));
+                    const uint32_t mw4[4] = {mb.x, mb.y, mb.z, mb.w};
+#pragma unroll
+                    for (int j = 0; j < 128; ++j) r[j] = ((mw4[j >> 5] >> (j & 31)) & 1u) ? r[j] : 0u;
+                    const float2 neg1 = make_float2(-1.0f, -1.0f);
+#pragma unroll
+                    for (int s2 = 32; s2 >= 1; s2 >>= 1) {          // strides 64 .. 2 in pairs of columns
+#pragma unroll
+                        for (int i = 0; i < 64; ++i)
+                            if ((i & s2) == 0) {
+                                const float2 a = make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+                                const float2 b = make_float2(__uint_as_float(r[2 * (i + s2)]), __uint_as_float(r[2 * (i + s2) + 1]));
+                                const float2 su = __fadd2_rn(a, b), di = __ffma2_rn(b, neg1, a);
+                                r[2 * i] = __float_as_uint(su.x); r[2 * i + 1] = __float_as_uint(su.y);
+                                r[2 * (i + s2)] = __float_as_uint(di.x); r[2 * (i + s2) + 1] = __float_as_uint(di.y);
+                            }
+                    }
+                    const float2 sc = make_float2(0.08838834764831845f, 0.08838834764831845f);    // 1 / sqrt(128)
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) {                  // stride 1, then the normalisation
+                        const float a = __uint_as_float(r[2 * i]), b = __uint_as_float(r[2 * i + 1]);
+                        const float2 o = __fmul2_rn(make_float2(a + b, a - b), sc);
+                        r[2 * i] = __float_as_uint(o.x);
+                        r[2 * i + 1] = __float_as_uint(o.y);
+                    }
+                }
+            }
 #pragma unroll
             for (int c0 = 0; c0 < CW; c0 += 32) {
                 const int col0 = n0 + cbase + c0;
                 if (col0 < p.N) {                      // uniform across the warp
                     const bool full = col0 + 32 <= p.N;
                     uint32_t *rc = &r[c0];
-                    if constexpr (BWD) {
+                    if constexpr (IHT128) {
+                        // already masked and transformed above
+                    } else if constexpr (BWD) {
                         // trust estimator: keep the gradient only where the forward mask trusts the element
                         const uint32_t mbits = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(
                                                             p.mask + (long long)row * (p.N >> 3) + (col0 >> 3)))
@@ -830,14 +868,17 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
 
 // Backward-pass contraction (Algorithm 2, lines 2 and 4): out[i][j] = mask[i][j] * sum_k a[i][k] b[j][k]
 // with bfloat16 operands a [I x Kc], b [J x Kc] (both dense, Kc contiguous) and binary32 output [I x J].
+// With fuse_iht128 (J % 128 == 0, I > 128, J > 128) the epilogue also applies the inverse Hadamard
+// transform on blocks of 128 columns and stores out_dtype; otherwise out is binary32.
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
-                            const uint8_t *mask, float *out, cudaStream_t st) {
+                            const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st) {
     if (I == 0 || J == 0) return QUEST_OK;
     GemmParams p;
     p.M = (int)I; p.N = (int)J; p.K = (int)(2 * Kc);
     p.sx = nullptr; p.sw = nullptr; p.rs_a = nullptr; p.rs_b = nullptr;
     p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
-    p.y = out; p.y_dtype = QUEST_F32; p.ldy = J; p.acc = nullptr; p.mask = mask;
+    p.y = out; p.y_dtype = out_dtype; p.ldy = J; p.acc = nullptr; p.mask = mask;
+    const int64_t esz = out_dtype == QUEST_F32 ? 4 : 2;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
     const bool wide = J > 128;
@@ -847,8 +888,13 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     if (s) return s;
     s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(b), J, 2 * Kc, pair ? 128 : wide ? 256 : 128);
     if (s) return s;
-    s = make_output_map(&tmY, out, I, J * 4, J * 4);
+    s = make_output_map(&tmY, out, I, J * esz, J * esz);
     if (s) return s;
+    if (fuse_iht128) {
+        if (!pair || J % 128 != 0) return QUEST_ERR_SHAPE;
+        return launch_gemm_bn<256, 3, true, true>(tmA, tmB, tmY, p, st);
+    }
+    if (out_dtype != QUEST_F32) return QUEST_ERR_DTYPE;
     if (pair) return launch_gemm_bn<256, 2, true, true>(tmA, tmB, tmY, p, st);
     if (wide) return launch_gemm_bn<256, 2, false, true>(tmA, tmB, tmY, p, st);
     return launch_gemm_bn<128, 2, false, true>(tmA, tmB, tmY, p, st);

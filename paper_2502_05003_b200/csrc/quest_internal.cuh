@@ -117,6 +117,6 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
                 int32_t *acc, cudaStream_t st);
 
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
-                            const uint8_t *mask, float *out, cudaStream_t st);
+                            const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st);
 
 }  // namespace quest
