@@ -178,7 +178,8 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
  *   dy                 device, [M x N] bfloat16, dense, 16-byte aligned
  *   M, N, K            M, N > 0 and multiples of 8; 32 <= K <= 16384, K % 32 == 0
  *   bits, had_block    as in the forward call that produced the codes
- *   xq, sx, mx         device: codes [M x K], scales [M], trust mask [M x K/8] of x (forward outputs)
+ *   xq, sx, mx         device: codes [M x K], scales [M], trust mask [M x K/8] of x (forward outputs);
+ *                      masks and sw 16-byte aligned, codes 4-byte aligned
  *   wq, sw, mw         the same for w ([N x K])
  *   dx, dw             device out: [M x K] and [N x K], dense, out_dtype (QUEST_F32 or QUEST_BF16),
  *                      16-byte aligned; either may be NULL to skip that gradient

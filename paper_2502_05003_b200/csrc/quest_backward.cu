@@ -27,62 +27,95 @@ __device__ __forceinline__ uint16_t bf16_bits(float v) {
     return *reinterpret_cast<uint16_t *>(&h);
 }
 
-// dy [M x N] bfloat16 -> a1 [M x N], a2 [N x M]; 32 x 32 tiles, block (32, 8).
+// dy [M x N] bfloat16 -> a1 [M x N] = dy * sw[n], a2 [N x M] = (dy * sx[m])^T, both rounded to bfloat16.
+// 64 x 64 tiles, 256 threads, 16-byte accesses on both sides (M and N are multiples of 8, so an
+// 8-element chunk is inside or outside the matrix as a whole).
 __global__ void __launch_bounds__(256)
 scale_dy_kernel(const uint16_t *__restrict__ dy, const float *__restrict__ sx, const float *__restrict__ sw,
                 int M, int N, uint16_t *__restrict__ a1, uint16_t *__restrict__ a2) {
-    __shared__ uint16_t tile[32][34];
+    __shared__ uint32_t tile[64][33];                          // [m][n pairs]; odd pitch keeps the transposed reads apart
     pdl_launch_dependents();
     pdl_wait();
-    const int m0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
-    const int tx = threadIdx.x, ty = threadIdx.y;
-    const int n = n0 + tx;
-    const float swn = n < N ? __ldg(sw + n) : 0.0f;
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    const int t = threadIdx.x;
+    const int chunk = t & 7;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int m = m0 + ty + 8 * i;
-        float v = 0.0f;
-        if (m < M && n < N) v = __uint_as_float((uint32_t)__ldg(dy + (long long)m * N + n) << 16);
-        if (m < M && n < N) a1[(long long)m * N + n] = bf16_bits(v * swn);
-        const float sxm = m < M ? __ldg(sx + m) : 0.0f;
-        tile[ty + 8 * i][tx] = bf16_bits(v * sxm);
+    for (int i = 0; i < 2; ++i) {
+        const int ml = (t >> 3) + 32 * i;
+        const int m = m0 + ml, n = n0 + chunk * 8;
+        uint32_t q[4] = {0u, 0u, 0u, 0u};
+        if (m < M && n < N) {
+            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(dy + (long long)m * N + n));
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+            const float sxm = __ldg(sx + m);
+            const float4 s0 = __ldg(reinterpret_cast<const float4 *>(sw + n));
+            const float4 s1 = __ldg(reinterpret_cast<const float4 *>(sw + n + 4));
+            const float swn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float lo = __uint_as_float(ww[j] << 16), hi = __uint_as_float(ww[j] & 0xFFFF0000u);
+                o[j] = (uint32_t)bf16_bits(lo * swn[2 * j]) | ((uint32_t)bf16_bits(hi * swn[2 * j + 1]) << 16);
+                q[j] = (uint32_t)bf16_bits(lo * sxm) | ((uint32_t)bf16_bits(hi * sxm) << 16);
+            }
+            *reinterpret_cast<uint4 *>(a1 + (long long)m * N + n) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) tile[ml][chunk * 4 + j] = q[j];
     }
     __syncthreads();
+    const uint16_t *t16 = reinterpret_cast<const uint16_t *>(&tile[0][0]);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int nn = n0 + ty + 8 * i, mm = m0 + tx;
-        if (nn < N && mm < M) a2[(long long)nn * M + mm] = tile[tx][ty + 8 * i];
+    for (int i = 0; i < 2; ++i) {
+        const int nl = (t >> 3) + 32 * i;
+        const int n = n0 + nl, m = m0 + chunk * 8;
+        if (n < N && m < M) {
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                o[j] = (uint32_t)t16[(chunk * 8 + 2 * j) * 66 + nl] | ((uint32_t)t16[(chunk * 8 + 2 * j + 1) * 66 + nl] << 16);
+            *reinterpret_cast<uint4 *>(a2 + (long long)n * M + m) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
     }
 }
 
-// packed codes [rows x K] -> ct [K x rows] bfloat16 grid values; 32 x 32 tiles, block (32, 8).
+// packed codes [rows x K] -> ct [K x rows] bfloat16 grid values c = 2k - (2^b - 1).
+// Tiles of 64 rows x 128 columns, 256 threads: a thread expands whole 32-bit code words into
+// shared memory, then the tile leaves transposed in 16-byte pieces (rows is a multiple of 8).
+template <int CB>
 __global__ void __launch_bounds__(256)
 codes_to_bf16_t_kernel(const uint8_t *__restrict__ codes, int bits, int rows, int K, uint16_t *__restrict__ ct) {
-    __shared__ uint16_t tile[32][34];
+    __shared__ __align__(16) uint16_t tile[128][72];           // [k][row], pitch 144 bytes
     pdl_launch_dependents();
     pdl_wait();
-    const int cb = container_bits(bits);
-    const int per = 8 / cb;
+    constexpr int PER = 32 / CB;                               // codes per word
+    constexpr int WPR = 128 / PER;                             // words per tile row
     const int L1 = (1 << bits) - 1;
-    const int r0 = blockIdx.y * 32, k0 = blockIdx.x * 32;
-    const int tx = threadIdx.x, ty = threadIdx.y;
-    const long long row_bytes = (long long)K * cb / 8;
+    const int r0 = blockIdx.y * 64, k0 = blockIdx.x * 128;
+    const int t = threadIdx.x;
+    const long long row_words = (long long)K * CB / 32;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int r = r0 + ty + 8 * i, k = k0 + tx;
-        float c = 0.0f;
-        if (r < rows && k < K) {
-            const int byte = __ldg(codes + r * row_bytes + k / per);
-            const int lev = (byte >> ((k % per) * cb)) & ((1 << cb) - 1);
-            c = (float)(2 * lev - L1);
+    for (int i = 0; i < (64 * WPR) / 256; ++i) {
+        const int w = t + 256 * i;
+        const int rl = w & 63, wl = w >> 6;                    // consecutive lanes: consecutive rows (conflict-free tile writes)
+        const int r = r0 + rl, k = k0 + wl * PER;
+        uint32_t word = 0;
+        const bool ok = r < rows && k < K;
+        if (ok) word = __ldg(reinterpret_cast<const uint32_t *>(codes) + r * row_words + (k0 / PER) + wl);
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int lev = (word >> (j * CB)) & ((1 << CB) - 1);
+            tile[wl * PER + j][rl] = ok ? bf16_bits((float)(2 * lev - L1)) : (uint16_t)0;    // |c| <= 255: exact
         }
-        tile[ty + 8 * i][tx] = bf16_bits(c);               // |c| <= 255: exact
     }
     __syncthreads();
+    const int chunk = t & 7;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const int kk = k0 + ty + 8 * i, rr = r0 + tx;
-        if (kk < K && rr < rows) ct[(long long)kk * rows + rr] = tile[tx][ty + 8 * i];
+        const int kl = (t >> 3) + 32 * i;
+        const int k = k0 + kl, r = r0 + chunk * 8;
+        if (k < K && r < rows)
+            *reinterpret_cast<uint4 *>(ct + (long long)k * rows + r) = *reinterpret_cast<const uint4 *>(&tile[kl][chunk * 8]);
     }
 }
 
@@ -235,20 +268,29 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
         return QUEST_ERR_HAD_BLOCK;
     if (out_dtype != QUEST_F32 && out_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
     auto al = [](const void *p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; };
-    if (!al(dy, 16) || !al(mx, 4) || !al(mw, 4) || (dx && !al(dx, 16)) || (dw && !al(dw, 16))) return QUEST_ERR_ALIGN;
+    if (!al(dy, 16) || !al(mx, 16) || !al(mw, 16) || !al(sw, 16) || !al(xq, 4) || !al(wq, 4) || (dx && !al(dx, 16)) ||
+        (dw && !al(dw, 16)))
+        return QUEST_ERR_ALIGN;
     if (!workspace || !al(workspace, 256) || workspace_bytes < quest_bwd_workspace_bytes(M, N, K))
         return QUEST_ERR_WORKSPACE;
     int s = check_device();
     if (s) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     BwdWorkspace ws = carve_bwd(workspace, M, N, K);
-    const dim3 blk(32, 8);
-    cudaError_t e = launch_pdl(scale_dy_kernel, dim3((unsigned)((N + 31) / 32), (unsigned)((M + 31) / 32)), blk, 0, st, 1,
+    cudaError_t e = launch_pdl(scale_dy_kernel, dim3((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64)), dim3(256), 0, st, 1,
                                reinterpret_cast<const uint16_t *>(dy), sx, sw, (int)M, (int)N, ws.a1, ws.a2);
     if (e != cudaSuccess) return cuda_fail(e);
+    auto codes_t = [&](const uint8_t *codes, int64_t rows, uint16_t *ct) -> cudaError_t {
+        const dim3 grid((unsigned)((K + 127) / 128), (unsigned)((rows + 63) / 64));
+        switch (container_bits(bits)) {
+            case 1: return launch_pdl(codes_to_bf16_t_kernel<1>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
+            case 2: return launch_pdl(codes_to_bf16_t_kernel<2>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
+            case 4: return launch_pdl(codes_to_bf16_t_kernel<4>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
+            default: return launch_pdl(codes_to_bf16_t_kernel<8>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
+        }
+    };
     if (dx) {
-        e = launch_pdl(codes_to_bf16_t_kernel, dim3((unsigned)((K + 31) / 32), (unsigned)((N + 31) / 32)), blk, 0, st, 1, wq, bits,
-                       (int)N, (int)K, ws.cwt);
+        e = codes_t(wq, N, ws.cwt);
         if (e != cudaSuccess) return cuda_fail(e);
         // line 2 and the mask of line 3: d1[m][k] = M_x[m][k] * sum_n a1[m][n] cwt[k][n]
         // (blocks of 128: the inverse transform is fused into the contraction's epilogue)
@@ -260,8 +302,7 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
         }
     }
     if (dw) {
-        e = launch_pdl(codes_to_bf16_t_kernel, dim3((unsigned)((K + 31) / 32), (unsigned)((M + 31) / 32)), blk, 0, st, 1, xq, bits,
-                       (int)M, (int)K, ws.cxt);
+        e = codes_t(xq, M, ws.cxt);
         if (e != cudaSuccess) return cuda_fail(e);
         // line 4 and the mask of line 5: d2[n][k] = M_w[n][k] * sum_m a2[n][m] cxt[k][m]
         if (had_block == 128 && N > 128 && K > 128) {
