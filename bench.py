@@ -452,6 +452,128 @@ def run_gpu(args, rank: int, world: int, local: int):
         dist.destroy_process_group()
 
 
+def run_backward(args, rank: int, world: int, local: int):
+    """Algorithm 2 on the same layer: `python bench.py --pass backward`.  One step = quest_linear_bwd
+    (both gradients) from the saved tensors of one forward call; same ring / graph / event method."""
+    import numpy as np
+    import torch
+
+    import paper_2502_05003_b200 as quest
+    from paper_2502_05003_b200 import synth
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    g = args.had_block
+    cfg = synth.config2()
+    M, K, N = TOKENS, HIDDEN, OUT
+    x = torch.from_numpy(cfg["x"]).view(torch.bfloat16).to(dev)
+    w = torch.from_numpy(cfg["w"]).view(torch.bfloat16).to(dev)
+    fwd = quest.quest_linear_fwd(x, w, BITS, g, 1.0)
+    rng = np.random.Generator(np.random.PCG64(7))
+    dy_bits = synth.f32_to_bf16_bits(rng.standard_normal((M, N), dtype=np.float32))
+    dy_host = torch.from_numpy(dy_bits).view(torch.bfloat16)
+    ws_bytes = quest.quest_bwd_workspace_bytes(M, N, K)
+
+    def make_set():
+        return {"dy": dy_host.to(dev), "dx": torch.empty((M, K), dtype=torch.bfloat16, device=dev),
+                "dw": torch.empty((N, K), dtype=torch.bfloat16, device=dev),
+                "ws": torch.empty(ws_bytes, dtype=torch.uint8, device=dev)}
+
+    set_bytes = M * N * 2 + (M + N) * K * 2 + ws_bytes
+    n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / set_bytes)))
+    ring = [make_set() for _ in range(n_sets)]
+
+    def step(i):
+        s = ring[i % n_sets]
+        quest.quest_linear_bwd(s["dy"], fwd, BITS, g, K, dx=s["dx"], dw=s["dw"], workspace=s["ws"])
+
+    def capture():
+        if args.no_graph:
+            return None
+        side = torch.cuda.Stream(device=dev)
+        g_ = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            for i in range(n_sets):
+                step(i)
+            side.synchronize()
+            with torch.cuda.graph(g_, stream=side):
+                for i in range(n_sets):
+                    step(i)
+        torch.cuda.synchronize()
+        return g_
+
+    def run_steps(k, graph):
+        if graph is None:
+            for i in range(k):
+                step(i)
+            return
+        for _ in range(k // n_sets):
+            graph.replay()
+        for i in range(k % n_sets):
+            step(i)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    graph = capture()
+    run_steps(n_sets, graph)
+    torch.cuda.synchronize()
+    steps = min(args.steps, 300)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        run_steps(steps, graph)
+        e1.record()
+        torch.cuda.synchronize()
+    elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3, world, dev)
+    if quest.quest_device_status() != 0:
+        raise RuntimeError("device status after the timed region")
+    quest.quest_stage_timing(True)
+    quest.quest_stage_times(reset=2)
+    staged = capture()
+    for r in range(30):
+        if staged is None:
+            step(r)
+        else:
+            staged.replay()
+        quest.quest_stage_times()
+    stage = quest.quest_stage_times(reset=2)
+    quest.quest_stage_timing(False)
+    stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+    if rank != 0:
+        return
+    peaks = load_peaks()
+    gemm_ms = stage_ms["gemm"]          # the second product (dL/dw) of the call; both have 2 M N K flops
+    tflops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12 if gemm_ms else None
+    # oracle: 64 rows of each gradient
+    from oracle import backward as ob
+    to_np = lambda t: t.cpu().numpy()
+    t0 = time.perf_counter()
+    rows = np.arange(64)
+    ob.backward(synth.bf16_bits_to_f32(dy_bits), to_np(fwd["xq"]), to_np(fwd["sx"]), to_np(fwd["mx"]), to_np(fwd["wq"]),
+                to_np(fwd["sw"]), to_np(fwd["mw"]), K, BITS, g, rows_x=rows, rows_w=rows)
+    o_dt = time.perf_counter() - t0
+    frac = (64.0 * N * K + 64.0 * M * K) / (2.0 * M * N * K)
+    line = {
+        "metric": "QuEST W4A4 linear bwd tokens/s", "value": M * steps * world / elapsed, "unit": UNIT, "n_gpus": world,
+        "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * elapsed / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": dict(workload_config(g), workload="config 2, Algorithm 2 (backward): dy[4096x2048] bf16 -> dx, dw bf16",
+                       l2="ring of %d buffer sets (%.0f MB) larger than L2" % (n_sets, n_sets * set_bytes / 1e6)),
+        "gpu_launches": 5 * steps, "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
+        "clocks": clocks.summary(),
+        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel<mode 3> (tcgen05 kind::f16 bf16, fused mask + inverse Hadamard)",
+                     "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": (tflops / peaks["bf16_tflops"]) if tflops else None,
+                     "peak_basis": "bf16 burst " + ("of measured" if peaks["_source"] == "measured" else "of fallback"),
+                     "traffic": None, "ms": gemm_ms},
+        "stage_ms": {"prepare": stage_ms["unpack"], "gemm_last": gemm_ms},
+        "cpu_baseline": {"value": M * frac / o_dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                         "sample": "64 rows of dL/dx and 64 rows of dL/dw (binary64 numpy), scaled by their share of the flops"},
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -460,6 +582,8 @@ def main():
     ap.add_argument("--impl", default="quest", choices=["quest", "reference"])
     ap.add_argument("--had-block", type=int, default=128)
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
+    ap.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward"],
+                    help="forward: Algorithm 1, the headline metric (default); backward: Algorithm 2 on the same layer")
     ap.add_argument("--ref-tokens", type=int, default=0,
                     help="token rows in the CPU oracle's bounded sample (0: the full 4096 for the "
                          "cpu_baseline leg; sized to about a minute in total for --impl reference)")
@@ -467,6 +591,9 @@ def main():
     rank, world, local = init_ranks(args.gpus)
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.which == "backward":
+        run_backward(args, rank, world, local)
         return
     run_gpu(args, rank, world, local)
 

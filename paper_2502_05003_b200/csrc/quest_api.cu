@@ -91,6 +91,10 @@ struct StageScope {
     }
 };
 
+// Stage brackets for translation units other than this one.
+void *stage_begin(int id, cudaStream_t st) { return new StageScope(id, st); }
+void stage_end(void *scope) { delete static_cast<StageScope *>(scope); }
+
 static bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
 static bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 

@@ -277,9 +277,15 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
     if (s) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     BwdWorkspace ws = carve_bwd(workspace, M, N, K);
+    struct Stage {                                   // RAII bracket for quest_stage_timing
+        void *h;
+        Stage(int id, cudaStream_t s_) : h(stage_begin(id, s_)) {}
+        ~Stage() { stage_end(h); }
+    };
+    Stage *prep = new Stage(QUEST_STAGE_UNPACK, st);   // operand preparation of the whole call up to the first product
     cudaError_t e = launch_pdl(scale_dy_kernel, dim3((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64)), dim3(256), 0, st, 1,
                                reinterpret_cast<const uint16_t *>(dy), sx, sw, (int)M, (int)N, ws.a1, ws.a2);
-    if (e != cudaSuccess) return cuda_fail(e);
+    if (e != cudaSuccess) { delete prep; return cuda_fail(e); }
     auto codes_t = [&](const uint8_t *codes, int64_t rows, uint16_t *ct) -> cudaError_t {
         const dim3 grid((unsigned)((K + 127) / 128), (unsigned)((rows + 63) / 64));
         switch (container_bits(bits)) {
@@ -291,7 +297,9 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
     };
     if (dx) {
         e = codes_t(wq, N, ws.cwt);
+        if (prep) { delete prep; prep = nullptr; }
         if (e != cudaSuccess) return cuda_fail(e);
+        Stage gemm_stage(QUEST_STAGE_GEMM, st);
         // line 2 and the mask of line 3: d1[m][k] = M_x[m][k] * sum_n a1[m][n] cwt[k][n]
         // (blocks of 128: the inverse transform is fused into the contraction's epilogue)
         if (had_block == 128 && M > 128 && K > 128) {
@@ -303,7 +311,9 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
     }
     if (dw) {
         e = codes_t(xq, M, ws.cxt);
+        if (prep) { delete prep; prep = nullptr; }
         if (e != cudaSuccess) return cuda_fail(e);
+        Stage gemm_stage(QUEST_STAGE_GEMM, st);
         // line 4 and the mask of line 5: d2[n][k] = M_w[n][k] * sum_m a2[n][m] cxt[k][m]
         if (had_block == 128 && N > 128 && K > 128) {
             if ((s = launch_gemm_bf16_masked(ws.a2, ws.cxt, N, K, M, mw, dw, out_dtype, true, st))) return s;

@@ -116,6 +116,10 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
                 int32_t *acc, cudaStream_t st);
 
+// Per-stage event timing (quest_stage_timing): bracket a stage of another translation unit.
+void *stage_begin(int id, cudaStream_t st);
+void stage_end(void *scope);
+
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
                             const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st);
 
