@@ -227,14 +227,15 @@ __device__ __forceinline__ void pin(uint32_t &v) { asm volatile("" : "+r"(v)::"m
 
 template <int BN, bool TWO>
 struct SmemLayout {
-    static constexpr int NSTAGES = TWO ? 5 : (BN == 256 ? 3 : STAGES);
+    static constexpr int NSTAGES = TWO ? 4 : (BN == 256 ? 3 : STAGES);   // four stages already saturate the MMA pipe
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_ROWS = TWO ? BN / 2 : BN;         // rows of B this CTA stages
     static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int BAR_OFFSET = NSTAGES * STAGE_BYTES;
-    static constexpr int STG_OFFSET = BAR_OFFSET;            // [8 warps][32 rows x 128 B] output staging
-    static constexpr int STG_BYTES = EPI_WARPS * 4096;
+    static constexpr int STG_OFFSET = BAR_OFFSET;            // [8 warps][SLABS][32 rows x 128 B] output staging
+    static constexpr int SLABS = (TWO || BN == 128) ? 2 : 1;
+    static constexpr int STG_BYTES = EPI_WARPS * SLABS * 4096;
     static constexpr int BAR_OFFSET2 = STG_OFFSET + STG_BYTES;
     static constexpr int SW_OFFSET = BAR_OFFSET2 + 256;      // [2][BN] column scales
     static constexpr int CB_OFFSET = SW_OFFSET + 2 * BN * 4; // [2][BN] column corrections (8-bit codes)
@@ -416,7 +417,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                    (p.ldy % (p.y_dtype == QUEST_BF16 ? 8 : 4) == 0));
         const bool vec_acc = p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
         const bool y_f32 = p.y_dtype == QUEST_F32;
-        uint8_t *slab = smem + L::STG_OFFSET + (warp - 2) * 4096;
+        uint8_t *slab_base = smem + L::STG_OFFSET + (warp - 2) * (L::SLABS * 4096);
+        int slab_count = 0;                            // slabs this warp has handed to TMA
         for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
             const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
             const int n0 = (tile / num_m) * BN;
@@ -558,9 +560,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             // j ^ (r & 7)), then one lane stores the slab with a TMA tile store, which clips
                             // at the matrix edges.  Binary32 fills a slab per 32 columns, bfloat16 per 64.
                             const int half = y_f32 ? 0 : ((c0 >> 5) & 1);
+                            uint8_t *slab = slab_base + (L::SLABS == 2 ? (slab_count & 1) * 4096 : 0);
                             if (half == 0) {
-                                // the previous store from this slab must have finished reading it
-                                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                                // the store that last used this slab must have finished reading it
+                                if (lane == 0) {
+                                    if (L::SLABS == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                                    else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                                }
                                 __syncwarp();
                             }
                             uint8_t *rowp = slab + lane * 128;
@@ -600,6 +606,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                         : "memory");
                                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                                 }
+                                ++slab_count;
                             }
                         } else if (row_ok) {
                             if (p.y_dtype == QUEST_BF16) {
