@@ -95,3 +95,56 @@ def gaussian_mse(alpha: float, bits: int) -> float:
         dPhi = Phi(hi) - Phi(lo)
         total += (dPhi - (xphi(hi) - xphi(lo))) + 2.0 * c * (phi(hi) - phi(lo)) + c * c * dPhi
     return total
+
+
+# ---- FP4 (E2M1) grid of Section 4.4 "The FP4 Format" -------------------------------------------
+
+E2M1_MAGNITUDES = (0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0)      # code magnitude index 0..7
+
+
+def fp4_grid() -> np.ndarray:
+    """The FP4 (E2M1) grid scaled to fit [-1, 1]: the 15 distinct values +-{0, .5, 1, 1.5, 2, 3, 4, 6} / 6."""
+    m = np.array(E2M1_MAGNITUDES[1:]) / 6.0
+    return np.concatenate([-m[::-1], [0.0], m])
+
+
+def gaussian_mse_points(alpha: float, points) -> float:
+    """E (xi - alpha * nearest(points, clip(xi, alpha) / alpha))^2 for xi ~ N(0,1), in closed form, for
+    any sorted grid `points` on [-1, 1] whose end points are -1 and +1 (cells end at the midpoints)."""
+    from math import erf, exp, pi, sqrt, inf
+
+    def Phi(v):
+        return 0.5 * (1.0 + erf(v / sqrt(2.0)))
+
+    def phi(v):
+        return 0.0 if v in (inf, -inf) else exp(-0.5 * v * v) / sqrt(2.0 * pi)
+
+    def xphi(v):
+        return 0.0 if v in (inf, -inf) else v * phi(v)
+
+    pts = [alpha * float(p) for p in points]
+    edges = [-inf] + [(pts[i] + pts[i + 1]) / 2 for i in range(len(pts) - 1)] + [inf]
+    total = 0.0
+    for k, c in enumerate(pts):
+        lo, hi = edges[k], edges[k + 1]
+        dPhi = Phi(hi) - Phi(lo)
+        total += (dPhi - (xphi(hi) - xphi(lo))) + 2.0 * c * (phi(hi) - phi(lo)) + c * c * dPhi
+    return total
+
+
+def project_fp4(xh: np.ndarray, alpha: float) -> dict:
+    """proj_alpha(x_h) with the FP4 grid by exhaustive nearest-point search (binary64).  Returns the
+    projected values, the per-row scale (xq = scale * v with v the E2M1 value in [-6, 6]), the
+    position t on the E2M1 value axis and the margin to the nearest cell boundary."""
+    xh = np.asarray(xh, dtype=np.float64)
+    rms = np.sqrt(np.mean(xh * xh, axis=1, keepdims=True))
+    safe = np.where(rms > 0, rms, 1.0)
+    clipped = np.clip(xh / safe, -alpha, alpha) / alpha
+    pts = fp4_grid()
+    k = np.argmin(np.abs(clipped[..., None] - pts[None, None, :]), axis=-1)
+    t = clipped * 6.0
+    vals = pts * 6.0
+    edges = (vals[:-1] + vals[1:]) / 2
+    margin = np.min(np.abs(t[..., None] - edges[None, None, :]), axis=-1)
+    return {"v": vals[k], "xq": alpha * rms * pts[k], "scale": (alpha * rms / 6.0)[:, 0], "rms": rms[:, 0],
+            "t": t, "margin": margin}

@@ -278,3 +278,121 @@ int qo_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t N,
     if (!acc_out) free(acc);
     return st;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * FP4 variant (Section 4.4, "The FP4 Format"): the rounding of Eq. 1 is replaced by rounding to
+ * the FP4 (E2M1) grid scaled to [-1, 1], alpha*_FP4 is the minimiser of the same Gaussian MSE with
+ * that grid, and the trust bound is the largest half-interval of the grid.
+ *
+ * E2M1 values: +-{0, 0.5, 1, 1.5, 2, 3, 4, 6}; a code is sign << 3 | magnitude index.  On the value
+ * axis t = x_h * 6 / (alpha* RMS) the grid points are the E2M1 values themselves, the largest
+ * interval is [4, 6], so T = 1 in these units.
+ * READING: ties between two neighbouring codes go to the even code (round-to-nearest-even of the
+ * E2M1 encoding); values beyond +-6 saturate; the sign of a value that rounds to zero is kept in
+ * the code (as a hardware conversion does).  PARITY UNPINNED by the paper.
+ * ------------------------------------------------------------------------------------------ */
+#define QO_ALPHA_STAR_FP4 2.9224751f
+
+static const float QO_E2M1[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+float qo_alpha_star_fp4(void) { return QO_ALPHA_STAR_FP4; }
+
+static int e2m1_index(float a) { /* a >= 0; interval midpoints, ties to the even index */
+    if (a <= 0.25f) return 0;
+    if (a < 0.75f) return 1;
+    if (a <= 1.25f) return 2;
+    if (a < 1.75f) return 3;
+    if (a <= 2.5f) return 4;
+    if (a < 3.5f) return 5;
+    if (a <= 5.0f) return 6;
+    return 7;
+}
+
+/* The E2M1 code (sign << 3 | magnitude index) of a position t on the value axis. */
+int qo_e2m1_code(float t) { return (signbit(t) ? 8 : 0) | e2m1_index(fabsf(t)); }
+
+/* Same rotation, RMS and outputs as qo_quantize; codes are E2M1 nibbles (element 0 in the low
+ * nibble), scales[r] = alpha*_FP4 RMS(x_h) / 6 so that xq_h = scale * E2M1 value. */
+int qo_quantize_fp4(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                    int had_block, float trust_factor,
+                    uint8_t *codes, float *scales, uint8_t *mask, float *t_out) {
+    if (!x || rows < 0 || cols <= 0 || ld < cols) return QO_BAD_ARG;
+    if (!is_pow2(had_block) || cols % had_block != 0) return QO_BAD_ARG;
+    if (dtype != 0 && dtype != 1) return QO_BAD_ARG;
+    if (cols % 8 != 0) return QO_BAD_ARG;
+    if (!(trust_factor >= 0.0f) || isinf(trust_factor)) return QO_BAD_ARG;
+    const float alpha = QO_ALPHA_STAR_FP4;
+    const float A = 6.0f / alpha;                           /* RMS-normalised value -> E2M1 value axis */
+    const float B = alpha / (6.0f * sqrtf((float)had_block));
+    const float h = trust_factor;                           /* largest half-interval of the grid: 1 */
+    int64_t p2 = 1;
+    while (p2 < cols) p2 *= 2;
+#pragma omp parallel
+    {
+        float *u = (float *)malloc(sizeof(float) * (size_t)cols);
+        float *tmp = (float *)malloc(sizeof(float) * (size_t)p2);
+#pragma omp for schedule(static)
+        for (int64_t r = 0; r < rows; ++r) {
+            if (dtype == 0) {
+                const float *xr = (const float *)x + r * ld;
+                for (int64_t e = 0; e < cols; ++e) u[e] = xr[e];
+            } else {
+                const uint16_t *xr = (const uint16_t *)x + r * ld;
+                for (int64_t e = 0; e < cols; ++e) u[e] = bf16_to_f32(xr[e]);
+            }
+            for (int64_t blk = 0; blk < cols; blk += had_block) qo_fwht_block(u + blk, had_block);
+            const float ss = sumsq_pairwise(u, cols, tmp, p2);
+            const float rms = sqrtf(ss / (float)cols);
+            const float inv = (rms > 0.0f) ? (A / rms) : 0.0f;
+            if (scales) scales[r] = rms * B;
+            uint8_t *cr = codes ? codes + r * (cols / 2) : 0;
+            uint8_t *mr = mask ? mask + r * (cols / 8) : 0;
+            if (cr) memset(cr, 0, (size_t)(cols / 2));
+            if (mr) memset(mr, 0, (size_t)(cols / 8));
+            for (int64_t e = 0; e < cols; ++e) {
+                const float t = u[e] * inv;
+                const int code = qo_e2m1_code(t);
+                const int m = code & 7;
+                const float v = signbit(t) ? -QO_E2M1[m] : QO_E2M1[m];
+                const int trusted = fabsf(t - v) <= h;
+                if (cr) cr[e / 2] |= (uint8_t)(code << ((e % 2) * 4));
+                if (mr && trusted) mr[e / 8] |= (uint8_t)(1u << (e % 8));
+                if (t_out) t_out[r * cols + e] = t;
+            }
+        }
+        free(u);
+        free(tmp);
+    }
+    return QO_OK;
+}
+
+/* Twice the E2M1 value of every code (an integer in [-12, 12]). */
+int qo_unpack_fp4_twice(const uint8_t *codes, int64_t rows, int64_t cols, int16_t *c2) {
+    if (!codes || !c2) return QO_BAD_ARG;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t e = 0; e < cols; ++e) {
+            const int code = (codes[r * (cols / 2) + e / 2] >> ((e % 2) * 4)) & 15;
+            const int two_v = (int)(2.0f * QO_E2M1[code & 7]);
+            c2[r * cols + e] = (int16_t)((code & 8) ? -two_v : two_v);
+        }
+    return QO_OK;
+}
+
+/* acc4[i][j] = sum_k (2 v_x[i][k]) (2 v_w[j][k]) = 4 * (xq_h wq_h^T)[i][j] / (sx[i] sw[j]), exact. */
+int qo_gemm_acc_fp4(const uint8_t *xq, const uint8_t *wq, int64_t M, int64_t N, int64_t K, int32_t *acc4) {
+    if (!xq || !wq || !acc4 || M < 0 || N < 0 || K <= 0) return QO_BAD_ARG;
+    int16_t *cx = (int16_t *)malloc(sizeof(int16_t) * (size_t)(M * K + 1));
+    int16_t *cw = (int16_t *)malloc(sizeof(int16_t) * (size_t)(N * K + 1));
+    qo_unpack_fp4_twice(xq, M, K, cx);
+    qo_unpack_fp4_twice(wq, N, K, cw);
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t s = 0;
+            for (int64_t k = 0; k < K; ++k) s += (int32_t)cx[i * K + k] * (int32_t)cw[j * K + k];
+            acc4[i * N + j] = (int32_t)s;
+        }
+    free(cx);
+    free(cw);
+    return QO_OK;
+}

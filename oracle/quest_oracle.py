@@ -57,6 +57,16 @@ def lib() -> ctypes.CDLL:
             L.qo_linear_fwd.restype = c_int
             L.qo_linear_fwd.argtypes = [vp, vp, c_int, i64, i64, i64, c_int, c_int, c_float,
                                         vp, vp, vp, vp, vp, vp, vp, vp]
+            L.qo_e2m1_code.restype = c_int
+            L.qo_e2m1_code.argtypes = [c_float]
+            L.qo_alpha_star_fp4.restype = c_float
+            L.qo_alpha_star_fp4.argtypes = []
+            L.qo_quantize_fp4.restype = c_int
+            L.qo_quantize_fp4.argtypes = [vp, c_int, i64, i64, i64, c_int, c_float, vp, vp, vp, vp]
+            L.qo_unpack_fp4_twice.restype = c_int
+            L.qo_unpack_fp4_twice.argtypes = [vp, i64, i64, vp]
+            L.qo_gemm_acc_fp4.restype = c_int
+            L.qo_gemm_acc_fp4.argtypes = [vp, vp, i64, i64, i64, vp]
             _lib = L
     return _lib
 
@@ -162,3 +172,49 @@ def linear_fwd(x: np.ndarray, w: np.ndarray, bits: int, had_block: int,
                              _ptr(out["wq"]), _ptr(out["sw"]), _ptr(out["mw"]))
     _check(st, "linear_fwd")
     return out
+
+
+# ---- FP4 (E2M1) grid variant ---------------------------------------------------------------------
+
+def alpha_star_fp4() -> float:
+    return float(lib().qo_alpha_star_fp4())
+
+
+def e2m1_code(t: float) -> int:
+    return int(lib().qo_e2m1_code(ctypes.c_float(t)))
+
+
+def quantize_fp4(x: np.ndarray, had_block: int, trust_factor: float = 1.0, debug: bool = False) -> dict:
+    """Rows of ``x`` -> E2M1 codes (two per byte), scales (xq_h = scale * E2M1 value), trust mask."""
+    x = np.ascontiguousarray(x)
+    rows, cols = x.shape
+    codes = np.zeros((rows, cols // 2), np.uint8)
+    scales = np.zeros(rows, np.float32)
+    mask = np.zeros((rows, cols // 8), np.uint8)
+    t = np.zeros((rows, cols), np.float32) if debug else None
+    _check(lib().qo_quantize_fp4(_ptr(x), _dtype_code(x), rows, cols, cols, had_block, ctypes.c_float(trust_factor),
+                                 _ptr(codes), _ptr(scales), _ptr(mask), _ptr(t)), "quantize_fp4")
+    out = {"codes": codes, "scales": scales, "mask": mask}
+    if debug:
+        out["t"] = t
+    return out
+
+
+def unpack_fp4_twice(codes: np.ndarray, cols: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    c2 = np.zeros((codes.shape[0], cols), np.int16)
+    _check(lib().qo_unpack_fp4_twice(_ptr(codes), codes.shape[0], cols, _ptr(c2)), "unpack_fp4")
+    return c2
+
+
+def gemm_acc_fp4(xq: np.ndarray, wq: np.ndarray, K: int) -> np.ndarray:
+    """acc4 = sum_k (2 v_x)(2 v_w): four times the product of the E2M1 values, exact int32."""
+    xq = np.ascontiguousarray(xq, dtype=np.uint8)
+    wq = np.ascontiguousarray(wq, dtype=np.uint8)
+    acc = np.zeros((xq.shape[0], wq.shape[0]), np.int32)
+    _check(lib().qo_gemm_acc_fp4(_ptr(xq), _ptr(wq), xq.shape[0], wq.shape[0], K, _ptr(acc)), "gemm_acc_fp4")
+    return acc
+
+
+def dequant_fp4(acc4: np.ndarray, sx: np.ndarray, sw: np.ndarray) -> np.ndarray:
+    return np.asarray(sx, np.float64)[:, None] * np.asarray(sw, np.float64)[None, :] * np.asarray(acc4, np.float64) / 4.0
