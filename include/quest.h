@@ -193,6 +193,33 @@ int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K, int bits, 
                      void *workspace, size_t workspace_bytes, void *stream);
 size_t quest_bwd_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
+/*
+ * FP4 variant -- Section 4.4, "The FP4 Format": the rounding of Eq. 1 is replaced by rounding to the
+ * FP4 (E2M1) grid +-{0, .5, 1, 1.5, 2, 3, 4, 6} scaled to [-1, 1], with alpha*_FP4 the minimiser of the
+ * same Gaussian MSE on that grid and the trust bound T its largest half-interval (times
+ * trust_factor).  Formats: codes are E2M1 nibbles (sign << 3 | magnitude index, two per byte,
+ * element 0 in the low nibble, rounded to nearest even and saturated by the hardware conversion);
+ * scale[row] = alpha*_FP4 RMS(x_h) / 6, so the dequantised element is scale * E2M1 value; masks as for
+ * the uniform grid.  The contraction runs on the int8 tensor cores with operands 2 v (exact):
+ * acc4[i][j] = 4 sum_k v_x v_w in int32, y = sx[i] sw[j] acc4 / 4.
+ * Arguments and rules are those of quest_quantize / quest_lowbit_gemm / quest_linear_fwd with
+ * bits = 4; cols (K) must be a multiple of 32.
+ */
+float quest_alpha_star_fp4(void);
+int quest_quantize_fp4(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
+                       int had_block, float trust_factor,
+                       uint8_t *codes, float *scales, uint8_t *mask, void *stream);
+int quest_lowbit_gemm_fp4(const uint8_t *xq, const float *sx, const uint8_t *wq, const float *sw,
+                          int64_t M, int64_t N, int64_t K,
+                          void *y, int y_dtype, int64_t ldy_elems, int32_t *acc4,
+                          void *workspace, size_t workspace_bytes, void *stream);
+int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                         int had_block, float trust_factor,
+                         void *y, int y_dtype,
+                         uint8_t *xq, float *sx, uint8_t *mx,
+                         uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
 /* Bytes of scratch quest_lowbit_gemm / quest_linear_fwd need (0 on invalid arguments). */
 size_t quest_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w);
 

@@ -235,3 +235,65 @@ def quest_linear_bwd(dy: torch.Tensor, fwd: dict, bits: int, had_block: int, K: 
                                       _p(workspace), workspace.numel(), _stream())
     _lib.check(st)
     return {"dx": dx, "dw": dw}
+
+
+# ---- FP4 (E2M1) grid variant: same calls with the FP4 rounding grid of Section 4.4 ---------------
+
+def quest_alpha_star_fp4() -> float:
+    return float(_lib.load().quest_alpha_star_fp4())
+
+
+def quest_quantize_fp4(x: torch.Tensor, had_block: int, trust_factor: float = 1.0):
+    """Rows of ``x`` -> (E2M1 codes uint8 [rows, cols/2], scales f32 [rows], mask uint8 [rows, cols/8])."""
+    _require_cuda(x)
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("quest_quantize_fp4: x must be 2-D with unit inner stride")
+    rows, cols = x.shape
+    codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty(rows, dtype=torch.float32, device=x.device)
+    mask = torch.empty((rows, cols // 8), dtype=torch.uint8, device=x.device)
+    _lib.check(_lib.load().quest_quantize_fp4(_p(x), _dtype_code(x), rows, cols, x.stride(0), had_block,
+                                              ctypes.c_float(trust_factor), _p(codes), _p(scales), _p(mask), _stream()))
+    return codes, scales, mask
+
+
+def quest_lowbit_gemm_fp4(xq, sx, wq, sw, K: int, out_dtype=torch.bfloat16, want_acc: bool = False, workspace=None):
+    """E2M1 codes -> (y [M, N], acc4 int32 [M, N] or None); acc4 is four times the value product."""
+    _require_cuda(xq, sx, wq, sw, workspace)
+    M, N = xq.shape[0], wq.shape[0]
+    y = torch.empty((M, N), dtype=out_dtype, device=xq.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=xq.device) if want_acc else None
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, 4, 4, xq.device)
+    _lib.check(_lib.load().quest_lowbit_gemm_fp4(_p(xq), _p(sx), _p(wq), _p(sw), M, N, K, _p(y), _dtype_code(y),
+                                                 y.stride(0), _p(acc), _p(workspace), workspace.numel(), _stream()))
+    return y, acc
+
+
+def quest_linear_fwd_fp4(x: torch.Tensor, w: torch.Tensor, had_block: int, trust_factor: float = 1.0,
+                         out_dtype=None, w_cached: dict = None, workspace: torch.Tensor = None) -> dict:
+    """Algorithm 1 with the FP4 grid: returns {"y", "xq", "sx", "mx", "wq", "sw", "mw"}."""
+    _require_cuda(x, w, workspace)
+    M, K = x.shape
+    dev = x.device
+    out = {}
+    if w_cached is not None:
+        out["wq"], out["sw"], out["mw"] = w_cached["wq"], w_cached["sw"], None
+        N = out["wq"].shape[0]
+    else:
+        N = w.shape[0]
+        out["wq"] = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+        out["sw"] = torch.empty(N, dtype=torch.float32, device=dev)
+        out["mw"] = torch.empty((N, K // 8), dtype=torch.uint8, device=dev)
+    out["xq"] = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+    out["sx"] = torch.empty(M, dtype=torch.float32, device=dev)
+    out["mx"] = torch.empty((M, K // 8), dtype=torch.uint8, device=dev)
+    y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, 4, 4, dev)
+    _lib.check(_lib.load().quest_linear_fwd_fp4(
+        _p(x), _p(w), _dtype_code(x), M, N, K, had_block, ctypes.c_float(trust_factor), _p(y), _dtype_code(y),
+        _p(out["xq"]), _p(out["sx"]), _p(out["mx"]), _p(out["wq"]), _p(out["sw"]), _p(out["mw"]),
+        1 if w_cached is not None else 0, _p(workspace), workspace.numel(), _stream()))
+    out["y"] = y
+    return out

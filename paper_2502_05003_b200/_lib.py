@@ -12,6 +12,7 @@ EXPORTS = (
     "quest_workspace_bytes", "quest_codes_bytes", "quest_alpha_star", "quest_device_status",
     "quest_status_string", "quest_last_cuda_error", "quest_stage_timing", "quest_stage_times",
     "quest_lowbit_gemm_static", "quest_linear_bwd", "quest_bwd_workspace_bytes",
+    "quest_alpha_star_fp4", "quest_quantize_fp4", "quest_lowbit_gemm_fp4", "quest_linear_fwd_fp4",
 )
 
 _lib = None
@@ -42,6 +43,14 @@ def load() -> ctypes.CDLL:
     L.quest_lowbit_gemm.argtypes = [vp, vp, ci, vp, vp, ci, i64, i64, i64, vp, ci, i64, vp, vp, sz, vp]
     L.quest_lowbit_gemm_static.restype = ci
     L.quest_lowbit_gemm_static.argtypes = [vp, vp, ci, vp, vp, ci, i64, i64, i64, vp, ci, i64, vp, vp]
+    L.quest_alpha_star_fp4.restype = cf
+    L.quest_alpha_star_fp4.argtypes = []
+    L.quest_quantize_fp4.restype = ci
+    L.quest_quantize_fp4.argtypes = [vp, ci, i64, i64, i64, ci, cf, vp, vp, vp, vp]
+    L.quest_lowbit_gemm_fp4.restype = ci
+    L.quest_lowbit_gemm_fp4.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, ci, i64, vp, vp, sz, vp]
+    L.quest_linear_fwd_fp4.restype = ci
+    L.quest_linear_fwd_fp4.argtypes = [vp, vp, ci, i64, i64, i64, ci, cf, vp, ci, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
     L.quest_linear_bwd.restype = ci
     L.quest_linear_bwd.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
     L.quest_bwd_workspace_bytes.restype = sz

@@ -313,4 +313,87 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
     return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits, bits, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);
 }
 
+// ---- FP4 (E2M1) grid variant (Section 4.4, "The FP4 Format") -----------------------------------
+
+float quest_alpha_star_fp4(void) { return alpha_star_fp4(); }
+
+int quest_quantize_fp4(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,
+                       int had_block, float trust_factor,
+                       uint8_t *codes, float *scales, uint8_t *mask, void *stream) {
+    int s = validate_quantize(x, dtype, rows, cols, ld_elems, 4, had_block, trust_factor, codes, mask);
+    if (s) return s;
+    if (cols % 32 != 0) return QUEST_ERR_SHAPE;
+    if ((s = check_device())) return s;
+    if (rows == 0) return QUEST_OK;
+    const QuantJob job = {x, rows, ld_elems, codes, scales, mask, nullptr, nullptr};
+    return launch_quantize(&job, 1, dtype, cols, 4, had_block, trust_factor, reinterpret_cast<cudaStream_t>(stream),
+                           GRID_FP4);
+}
+
+int quest_lowbit_gemm_fp4(const uint8_t *xq, const float *sx, const uint8_t *wq, const float *sw,
+                          int64_t M, int64_t N, int64_t K,
+                          void *y, int y_dtype, int64_t ldy_elems, int32_t *acc4,
+                          void *workspace, size_t workspace_bytes, void *stream) {
+    int s = validate_gemm_shape(M, N, K, 4, 4);
+    if (s) return s;
+    if (M == 0 || N == 0) return QUEST_OK;
+    if (!xq || !wq) return QUEST_ERR_NULL;
+    if (!y && !acc4) return QUEST_ERR_NULL;
+    if (y && (!sx || !sw)) return QUEST_ERR_NULL;
+    if (y) {
+        if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+        if (ldy_elems < N) return QUEST_ERR_SHAPE;
+        if (!aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    }
+    if (!aligned(xq, 16) || !aligned(wq, 16) || (acc4 && !aligned(acc4, 4))) return QUEST_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, 4, 4))
+        return QUEST_ERR_WORKSPACE;
+    if ((s = check_device())) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    Workspace ws = carve_workspace(workspace, M, N, K);
+    {
+        StageScope scope(QUEST_STAGE_UNPACK, st);
+        if ((s = launch_unpack(xq, 4, M, K, ws.a8, nullptr, st, GRID_FP4))) return s;
+        if ((s = launch_unpack(wq, 4, N, K, ws.b8, nullptr, st, GRID_FP4))) return s;
+    }
+    StageScope scope(QUEST_STAGE_GEMM, st);
+    return launch_gemm(ws.a8, ws.b8, nullptr, nullptr, 4, 4, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc4, st, GRID_FP4);
+}
+
+int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                         int had_block, float trust_factor,
+                         void *y, int y_dtype,
+                         uint8_t *xq, float *sx, uint8_t *mx,
+                         uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                         void *workspace, size_t workspace_bytes, void *stream) {
+    if (!y || !xq || !sx || !wq || !sw) return QUEST_ERR_NULL;
+    if (!w_is_cached && !w) return QUEST_ERR_NULL;
+    if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+    int s = validate_gemm_shape(M, N, K, 4, 4);
+    if (s) return s;
+    if ((s = validate_quantize(x, dtype, M, K, K, 4, had_block, trust_factor, xq, mx))) return s;
+    if (!w_is_cached && (s = validate_quantize(w, dtype, N, K, K, 4, had_block, trust_factor, wq, mw))) return s;
+    if (!aligned(wq, 16) || !aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, 4, 4))
+        return QUEST_ERR_WORKSPACE;
+    if ((s = check_device())) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    Workspace ws = carve_workspace(workspace, M, N, K);
+    const QuantJob jx = {x, M, K, xq, sx, mx, ws.a8, nullptr};
+    if (w_is_cached) {
+        {
+            StageScope scope(QUEST_STAGE_QUANT_X, st);
+            if ((s = launch_quantize(&jx, 1, dtype, K, 4, had_block, trust_factor, st, GRID_FP4))) return s;
+        }
+        StageScope scope(QUEST_STAGE_UNPACK, st);
+        if ((s = launch_unpack(wq, 4, N, K, ws.b8, nullptr, st, GRID_FP4))) return s;
+    } else {
+        StageScope scope(QUEST_STAGE_QUANT_X, st);
+        const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, ws.b8, nullptr}};
+        if ((s = launch_quantize(jobs, 2, dtype, K, 4, had_block, trust_factor, st, GRID_FP4))) return s;
+    }
+    StageScope scope(QUEST_STAGE_GEMM, st);
+    return launch_gemm(ws.a8, ws.b8, nullptr, nullptr, 4, 4, sx, sw, M, N, K, y, y_dtype, N, nullptr, st, GRID_FP4);
+}
+
 }  // extern "C"

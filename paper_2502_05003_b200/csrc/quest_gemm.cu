@@ -57,6 +57,7 @@ struct GemmParams {
     const int32_t *rs_b;   // row sums of the B operand values (nullable)
     int mul;               // acc' = (mul*acc + ca*rs_a[i] + cb*rs_b[j] + ck) >> sh   (exact)
     int ca, cb, ck, sh;
+    int ysh;               // y carries an extra exact factor 2^-ysh (FP4 grid: operands are twice the E2M1 values)
     void *y;
     int y_dtype;
     long long ldy;
@@ -441,6 +442,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool fold = !CORR && !p.acc;
             float sxr = (!BWD && row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
             if (fold) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.sh) << 23));
+            if (p.ysh) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.ysh) << 23));
             int rsa = 0;
             if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
             ok = mbar_wait(smem_u32(&tfull_bar[buf]), bphase, abort_flag, p.status, ST_EPILOGUE);
@@ -691,6 +693,22 @@ __global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits,
     }
 }
 
+// E2M1 codes -> int8 operand values 2 v, 32 elements per thread.
+__global__ void unpack_fp4_kernel(const uint8_t *__restrict__ codes, long long n_groups, int8_t *__restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n_groups;
+         g += (long long)gridDim.x * blockDim.x) {
+        const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + g);
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+        uint32_t o[8];
+        fp4_operand_from_code_words(w, o);
+        uint4 *dst = reinterpret_cast<uint4 *>(out + g * 32);
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
 // Row sums of an int8 matrix [rows x K]: one warp per row.
 __global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, int K, int32_t *__restrict__ out) {
     pdl_launch_dependents();
@@ -801,13 +819,17 @@ Workspace carve_workspace(void *base, int64_t M, int64_t N, int64_t K) {
 }
 
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out, int32_t *rowsum,
-                  cudaStream_t st) {
+                  cudaStream_t st, int grid) {
     if (rows == 0) return QUEST_OK;
     const long long n_groups = rows * K / 32;
     const int threads = 256;
     long long blocks = (n_groups + threads - 1) / threads;
     if (blocks > 148 * 16) blocks = 148 * 16;
     cudaError_t e;
+    if (grid == GRID_FP4) {
+        e = launch_pdl(unpack_fp4_kernel, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, n_groups, out);
+        return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+    }
     switch (container_bits(bits)) {
         case 1: e = launch_pdl(unpack_codes_kernel<1>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
         case 2: e = launch_pdl(unpack_codes_kernel<2>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
@@ -829,7 +851,7 @@ int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cu
 int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
                 int bits_x, int bits_w, const float *sx, const float *sw,
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
-                int32_t *acc, cudaStream_t st) {
+                int32_t *acc, cudaStream_t st, int grid) {
     if (M == 0 || N == 0) return QUEST_OK;
     // operand value v relates to the grid value c by v = 2^(7-b) c below 8 bits and c = 2v + 1 at 8 bits
     const bool x8 = bits_x == 8, w8 = bits_w == 8;
@@ -840,6 +862,10 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
     else if (x8 && w8) { p.mul = 4; p.ca = 2; p.cb = 2; p.ck = (int)K; p.sh = 0; }
     else if (x8) { p.mul = 2; p.ca = 0; p.cb = 1; p.ck = 0; p.sh = 7 - bits_w; }   // 2 sum v_x op_w + sum op_w
     else { p.mul = 2; p.ca = 1; p.cb = 0; p.ck = 0; p.sh = 7 - bits_x; }
+    p.ysh = 0;
+    if (grid == GRID_FP4) {    // operands are 2 v: acc = 4 sum v_x v_w is reported as is, y takes the factor 1/4
+        p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; p.ysh = 2;
+    }
     p.rs_a = p.ca ? rs_a : nullptr;                      // row sums of the x operand bytes
     p.rs_b = p.cb ? rs_b : nullptr;                      // row sums of the w operand bytes
     p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr;
@@ -883,7 +909,7 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     GemmParams p;
     p.M = (int)I; p.N = (int)J; p.K = (int)(2 * Kc);
     p.sx = nullptr; p.sw = nullptr; p.rs_a = nullptr; p.rs_b = nullptr;
-    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
+    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; p.ysh = 0;
     p.y = out; p.y_dtype = out_dtype; p.ldy = J; p.acc = nullptr; p.mask = mask;
     const int64_t esz = out_dtype == QUEST_F32 ? 4 : 2;
     p.status = device_status_word();

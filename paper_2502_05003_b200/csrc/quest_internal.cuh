@@ -36,9 +36,14 @@ struct QuantConsts {
     float top;     // 2^b-1: highest level
     float A;       // (2^b-1)/(2 alpha*): RMS-normalised value -> level-axis slope
     float B;       // alpha*/((2^b-1) sqrt(g)): RMS of the un-normalised rotation -> scale
-    float h;       // trust_factor/2: trust bound in level steps
+    float h;       // trust_factor/2: trust bound in level steps (FP4 grid: trust_factor, in E2M1 value units)
 };
 QuantConsts make_quant_consts(int bits, int had_block, float trust_factor);
+
+// Rounding grids: the uniform zero-free grid of Eq. 1, or the FP4 (E2M1) grid of Section 4.4.
+enum { GRID_UNIFORM = 0, GRID_FP4 = 1 };
+// alpha*_FP4: minimiser of the Gaussian quantisation MSE on the E2M1 grid scaled to [-1, 1].
+__host__ __device__ inline float alpha_star_fp4() { return 2.9224751f; }
 
 // Operand layout of the int8 tensor-core contraction inside the workspace.
 struct Workspace {
@@ -107,14 +112,14 @@ struct QuantJob {
 };
 // Up to two tensors with the same row length, dtype and parameters share one launch.
 int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
-                    float trust_factor, cudaStream_t st);
+                    float trust_factor, cudaStream_t st, int grid = GRID_UNIFORM);
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out,
-                  int32_t *rowsum, cudaStream_t st);
+                  int32_t *rowsum, cudaStream_t st, int grid = GRID_UNIFORM);
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st);
 int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
                 int bits_x, int bits_w, const float *sx, const float *sw,
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
-                int32_t *acc, cudaStream_t st);
+                int32_t *acc, cudaStream_t st, int grid = GRID_UNIFORM);
 
 // Per-stage event timing (quest_stage_timing): bracket a stage of another translation unit.
 void *stage_begin(int id, cudaStream_t st);

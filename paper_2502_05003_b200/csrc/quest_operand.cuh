@@ -86,6 +86,34 @@ __device__ __forceinline__ void operand_from_code_words(const uint32_t (&w)[CB],
     }
 }
 
+// FP4 (E2M1) codes: sign << 3 | magnitude index m, values +-{0, .5, 1, 1.5, 2, 3, 4, 6}.
+// Twice the magnitude is an integer: m for m < 2, else (2 + (m & 1)) << ((m >> 1) - 1).
+__device__ __forceinline__ int e2m1_twice_magnitude(int m) {
+    const int e = m >> 1;
+    return e ? (2 + (m & 1)) << (e - 1) : m;
+}
+__device__ __forceinline__ float e2m1_value(int code) {
+    const int m = code & 7, e = m >> 1;
+    const float mag = e ? __uint_as_float(((uint32_t)(126 + e) << 23) | ((uint32_t)(m & 1) << 22)) : 0.5f * (float)m;
+    return (code & 8) ? -mag : mag;
+}
+// 32 consecutive E2M1 codes (4 words, element 0 in the low nibble) -> 32 operand bytes 2 v (|2v| <= 12).
+__device__ __forceinline__ void fp4_operand_from_code_words(const uint32_t (&w)[4], uint32_t (&o)[8]) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int e = q * 4 + j;
+            const int code = (w[e >> 3] >> ((e & 7) * 4)) & 15;
+            const int mag2 = e2m1_twice_magnitude(code & 7);
+            const int val = (code & 8) ? -mag2 : mag2;
+            acc |= (uint32_t)(val & 0xFF) << (8 * j);
+        }
+        o[q] = acc;
+    }
+}
+
 // Sum of the four signed bytes of a word.
 __device__ __forceinline__ int sum_bytes_s8(uint32_t w) { return __dp4a((int)w, 0x01010101, 0); }
 

@@ -13,6 +13,17 @@
 
 namespace quest {
 
+QuantConsts make_quant_consts_fp4(int had_block, float trust_factor) {
+    QuantConsts c;
+    const float alpha = alpha_star_fp4();
+    c.c0 = 0.0f;
+    c.top = 6.0f;
+    c.A = 6.0f / alpha;                                   // RMS-normalised value -> E2M1 value axis
+    c.B = alpha / (6.0f * sqrtf((float)had_block));
+    c.h = trust_factor;                                   // largest half-interval of the grid: 1 value unit
+    return c;
+}
+
 QuantConsts make_quant_consts(int bits, int had_block, float trust_factor) {
     QuantConsts c;
     const int L1 = (1 << bits) - 1;
@@ -156,12 +167,28 @@ struct QuantArgs {
     int S, R;
 };
 
+// Eight positions on the E2M1 value axis -> eight 4-bit codes in one word (element 0 in the low
+// nibble), rounded to nearest even and saturated by the hardware conversion.
+__device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+        : "=r"(out)
+        : "f"(t[0]), "f"(t[1]), "f"(t[2]), "f"(t[3]), "f"(t[4]), "f"(t[5]), "f"(t[6]), "f"(t[7]));
+    return out;
+}
+
 // Everything after the load: rotation from stride s_start downwards (larger strides already
 // applied by the caller), RMS, projection, trust test, packing and stores for the E elements this
 // thread holds.  GFULL: had_block >= E, so every in-register stage runs.  FAST: the common case
 // fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
 // one warp, every output requested, no row sums -- so that no per-row branch or loop remains.
-template <int CB, int E, bool GFULL, bool FAST>
+template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
                                                      int s_start) {
@@ -286,6 +313,28 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
         for (int g32 = 0; g32 < E / 32; ++g32) {
             uint32_t kb[32];                                    // MAGIC_BITS + level
             uint32_t mbits = 0;
+            uint32_t w[CB];
+            if constexpr (GRID == GRID_FP4) {
+                // FP4 grid (Section 4.4): t = u * inv on the E2M1 value axis, hardware rounding to E2M1,
+                // trusted = |t - value| <= trust_factor (the largest half-interval is one value unit)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float t[8];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        t[2 * j] = __fmul_rn(v[g32 * 16 + q * 4 + j].x, inv);
+                        t[2 * j + 1] = __fmul_rn(v[g32 * 16 + q * 4 + j].y, inv);
+                    }
+                    const uint32_t cw = cvt_e2m1x8(t);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float val = e2m1_value((int)((cw >> (4 * j)) & 15u));
+                        const bool trusted = fabsf(__fsub_rn(t[j], val)) <= hh;
+                        mbits |= (trusted ? 1u : 0u) << (q * 8 + j);
+                    }
+                    w[q] = cw;
+                }
+            } else {
 #pragma unroll
             for (int i = 15; i >= 0; --i) {
                 const float2 t = __ffma2_rn(v[g32 * 16 + i], inv2, c02);
@@ -303,6 +352,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 kb[2 * i + 1] = __float_as_uint(km.y);
             }
             mbits = ~mbits;
+            }
             if (FAST || tn.mask)
                 reinterpret_cast<uint32_t *>(tn.mask + row * (long long)(cols >> 3))[tr * (E / 32) + g32] = mbits;
 
@@ -311,13 +361,14 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
             uint32_t magic_sum = 0;
 #pragma unroll
             for (int j = 0; j < PER; ++j) magic_sum += QUEST_MAGIC_BITS << (CB * j);
-            uint32_t w[CB];
+            if constexpr (GRID != GRID_FP4) {
 #pragma unroll
-            for (int q = 0; q < CB; ++q) {
-                uint32_t acc = 0;
+                for (int q = 0; q < CB; ++q) {
+                    uint32_t acc = 0;
 #pragma unroll
-                for (int j = PER - 1; j >= 0; --j) acc = (acc << CB) + kb[q * PER + j];
-                w[q] = acc - magic_sum;
+                    for (int j = PER - 1; j >= 0; --j) acc = (acc << CB) + kb[q * PER + j];
+                    w[q] = acc - magic_sum;
+                }
             }
             if (FAST || tn.codes) {
                 uint8_t *dst = tn.codes + row * (long long)(cols * CB / 8) + ((long long)tr * (E / 32) + g32) * (4 * CB);
@@ -334,7 +385,8 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
             }
             if (FAST || tn.op8) {
                 uint32_t o[8];
-                operand_from_code_words<CB>(w, a.bits, o);
+                if constexpr (GRID == GRID_FP4) fp4_operand_from_code_words(w, o);
+                else operand_from_code_words<CB>(w, a.bits, o);
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -362,7 +414,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
     }
 }
 
-template <bool BF16, int CB, int E>
+template <bool BF16, int CB, int E, int GRID = GRID_UNIFORM>
 __global__ void __launch_bounds__(E == 64 ? 256 : 512)
 quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
     extern __shared__ float xsm[];                 // [E][blockDim.x] exchange, then [warps] partial sums
@@ -405,7 +457,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
 #pragma unroll
         for (int i = 0; i < H; ++i) v[i] = make_float2(0.0f, 0.0f);
     }
-    rotate_project_store<CB, E, false, false>(v, a, tn, active, row, tr, r_local, xsm, a.had_block >> 1);
+    rotate_project_store<CB, E, false, false, GRID>(v, a, tn, active, row, tr, r_local, xsm, a.had_block >> 1);
 }
 
 // Streaming variant for bfloat16 rows (E = 64, had_block >= 64): a persistent grid in which every
@@ -528,6 +580,17 @@ static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cuda
     return cudaGetLastError();
 }
 
+// FP4 grid: 4-bit containers only.
+template <bool BF16, int E>
+static cudaError_t launch_rows_fp4(dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
+    if (smem > 48 * 1024) {
+        cudaError_t e_ = cudaFuncSetAttribute(quantize_rows_kernel<BF16, 4, E, GRID_FP4>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
+        if (e_ != cudaSuccess) return e_;
+    }
+    return launch_pdl(quantize_rows_kernel<BF16, 4, E, GRID_FP4>, grid, dim3(threads), smem, st, 1, a);
+}
+
 template <int E, bool FAST>
 static cudaError_t launch_stream(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                  int total_groups, int exchange_bytes) {
@@ -551,13 +614,15 @@ static cudaError_t launch_stream(int cb, int grid, int threads, size_t smem, cud
 }  // namespace
 
 int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
-                    float trust_factor, cudaStream_t st) {
-    const QuantConsts qc = make_quant_consts(bits, had_block, trust_factor);
+                    float trust_factor, cudaStream_t st, int grid_kind) {
+    const QuantConsts qc = grid_kind == GRID_FP4 ? make_quant_consts_fp4(had_block, trust_factor)
+                                                 : make_quant_consts(bits, had_block, trust_factor);
+    if (grid_kind == GRID_FP4 && cols % 32 != 0) return QUEST_ERR_SHAPE;
     const int cb = container_bits(bits);
     if (cols % 32 == 0) {
         // streaming kernel with 32 elements per thread (64 registers, twice the resident warps) measured
         // faster than 64 per thread for rows up to 4096 elements; wider rows keep 64 per thread
-        const bool stream32 = dtype == QUEST_BF16 && had_block >= 64 && cols <= 4096;
+        const bool stream32 = grid_kind == GRID_UNIFORM && dtype == QUEST_BF16 && had_block >= 64 && cols <= 4096;
         const int E = (cols % 64 == 0 && !stream32) ? 64 : 32;
         const int T = (int)(cols / E);
         int S;
@@ -587,7 +652,14 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = S; a.R = R;
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
-            if ((E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64) {
+            if (grid_kind == GRID_FP4) {
+                if (E == 64)
+                    e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 64>(grid, threads, smem, st, a)
+                                            : launch_rows_fp4<false, 64>(grid, threads, smem, st, a);
+                else
+                    e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 32>(grid, threads, smem, st, a)
+                                            : launch_rows_fp4<false, 32>(grid, threads, smem, st, a);
+            } else if ((E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64) {
                 // persistent streaming kernel: as many CTAs as fit on the device, each looping over groups
                 const int exchange = (int)((smem + 15) / 16 * 16);
                 const size_t smem2 = (size_t)exchange + 2 * (size_t)threads * (2 * E + 16);

@@ -141,3 +141,13 @@ def test_backward_argument_errors(lib):
     assert lib.quest_bwd_workspace_bytes(4096, 2048, 2048) >= (2 * 4096 * 2048 + 2048 * 2048 + 4096 * 2048) * 2 + \
         (4096 + 2048) * 2048 * 4
     assert lib.quest_bwd_workspace_bytes(60, 64, 128) == 0
+
+
+def test_fp4_entry_points_validate_on_the_host(lib):
+    assert abs(lib.quest_alpha_star_fp4() - 2.9224751) < 1e-6
+    q = lambda **kw: lib.quest_quantize_fp4(kw.get("x", FAKE), kw.get("dtype", 1), kw.get("rows", 4), kw.get("cols", 128),
+                                            kw.get("ld", 128), kw.get("g", 128), F(kw.get("trust", 1.0)), FAKE, FAKE, FAKE, None)
+    assert q(x=None) == 1 and q(dtype=9) == 5 and q(cols=40, ld=40, g=8) == 2 and q(g=48) == 4 and q(trust=-1.0) == 7
+    g = lambda **kw: lib.quest_lowbit_gemm_fp4(kw.get("xq", FAKE), FAKE, FAKE, FAKE, kw.get("M", 64), 64, kw.get("K", 128),
+                                               FAKE, kw.get("yd", 1), 64, None, kw.get("ws", FAKE), kw.get("wsb", 1 << 20), None)
+    assert g(xq=None) == 1 and g(K=100) == 2 and g(yd=4) == 5 and g(ws=None) == 8 and g(wsb=8) == 8
