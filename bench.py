@@ -2,11 +2,15 @@
 """Benchmark of the QuEST quantized-linear forward hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--had-block G]
+                    [--no-graph] [--pass backward]
 
 One "step" is one pass of the whole path (Algorithm 1: quantize X, quantize W, low-bit GEMM with
 the dequantising epilogue) through the C ABI call ``quest_linear_fwd`` on the 1.6B-scale layer:
 X[4096 x 2048] bf16, W[2048 x 2048] bf16, b = 4, Hadamard block 128 (seeded synthetic data).
-The step rotates over a ring of buffer sets larger than L2, so every step streams from HBM.
+The step rotates over a ring of buffer sets larger than L2, so every step streams from HBM, and the
+timed steps are replayed from a CUDA graph holding one pass over the ring (``--no-graph``: direct
+launches), because the host cannot launch a step of a few tens of microseconds fast enough.
+``--pass backward`` times Algorithm 2 (``quest_linear_bwd``) on the same layer instead.
 
 Prints ONE JSON line (rank 0).  ``value`` is tokens/s with inputs resident in HBM; ``e2e`` is the
 same metric with the host->device copy of X and W and the device->host copy of y inside the
