@@ -326,11 +326,19 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                         t[2 * j + 1] = __fmul_rn(v[g32 * 16 + q * 4 + j].y, inv);
                     }
                     const uint32_t cw = cvt_e2m1x8(t);
+                    if (hh >= 1.0f) {
+                        // every element inside the grid is within one value unit of its point (exactly, the
+                        // difference being exact); only saturated elements can fail: |t| - 6 > trust_factor
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float val = e2m1_value((int)((cw >> (4 * j)) & 15u));
-                        const bool trusted = fabsf(__fsub_rn(t[j], val)) <= hh;
-                        mbits |= (trusted ? 1u : 0u) << (q * 8 + j);
+                        for (int j = 0; j < 8; ++j)
+                            mbits |= (__fsub_rn(fabsf(t[j]), 6.0f) <= hh ? 1u : 0u) << (q * 8 + j);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float val = e2m1_value((int)((cw >> (4 * j)) & 15u));
+                            const bool trusted = fabsf(__fsub_rn(t[j], val)) <= hh;
+                            mbits |= (trusted ? 1u : 0u) << (q * 8 + j);
+                        }
                     }
                     w[q] = cw;
                 }
@@ -468,7 +476,7 @@ quantize_rows_kernel(const __grid_constant__ QuantArgs a) {
 // (source size 0), so reads need no predicate.  The first butterfly stage (stride had_block/2)
 // pairs this thread with thread tid ^ dist0 of the same row; both read both raw slots from shared
 // memory, so that stage needs no shuffles.
-template <int CB, int E, bool FAST>
+template <int CB, int E, bool FAST, int GRID = GRID_UNIFORM>
 __global__ void __launch_bounds__(256, E == 64 ? 2 : 4)
 quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, int exchange_bytes) {
     constexpr int H = E / 2;
@@ -553,7 +561,7 @@ quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, in
 #pragma unroll
             for (int q = 0; q < E / 8; ++q) widen(own[q], &v[q * 4]);
         }
-        rotate_project_store<CB, E, true, FAST>(v, a, tn, active, row, tr, r_local, xsm, s_start);
+        rotate_project_store<CB, E, true, FAST, GRID>(v, a, tn, active, row, tr, r_local, xsm, s_start);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
@@ -591,6 +599,16 @@ static cudaError_t launch_rows_fp4(dim3 grid, int threads, size_t smem, cudaStre
     return launch_pdl(quantize_rows_kernel<BF16, 4, E, GRID_FP4>, grid, dim3(threads), smem, st, 1, a);
 }
 
+template <int E>
+static cudaError_t launch_stream_fp4(int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                                     int total_groups, int exchange_bytes) {
+    cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<4, E, false, GRID_FP4>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    if (e_ != cudaSuccess) return e_;
+    return launch_pdl(quantize_stream_kernel<4, E, false, GRID_FP4>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a,
+                      total_groups, exchange_bytes);
+}
+
 template <int E, bool FAST>
 static cudaError_t launch_stream(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                  int total_groups, int exchange_bytes) {
@@ -622,7 +640,7 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
     if (cols % 32 == 0) {
         // streaming kernel with 32 elements per thread (64 registers, twice the resident warps) measured
         // faster than 64 per thread for rows up to 4096 elements; wider rows keep 64 per thread
-        const bool stream32 = grid_kind == GRID_UNIFORM && dtype == QUEST_BF16 && had_block >= 64 && cols <= 4096;
+        const bool stream32 = dtype == QUEST_BF16 && had_block >= 64 && cols <= 4096;
         const int E = (cols % 64 == 0 && !stream32) ? 64 : 32;
         const int T = (int)(cols / E);
         int S;
@@ -652,14 +670,15 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = S; a.R = R;
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
-            if (grid_kind == GRID_FP4) {
+            const bool streaming = (E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64;
+            if (grid_kind == GRID_FP4 && !streaming) {
                 if (E == 64)
                     e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 64>(grid, threads, smem, st, a)
                                             : launch_rows_fp4<false, 64>(grid, threads, smem, st, a);
                 else
                     e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 32>(grid, threads, smem, st, a)
                                             : launch_rows_fp4<false, 32>(grid, threads, smem, st, a);
-            } else if ((E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64) {
+            } else if (streaming) {
                 // persistent streaming kernel: as many CTAs as fit on the device, each looping over groups
                 const int exchange = (int)((smem + 15) / 16 * 16);
                 const size_t smem2 = (size_t)exchange + 2 * (size_t)threads * (2 * E + 16);
@@ -674,7 +693,10 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                     const QuantTensor &t = a.t[j];
                     if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum)) fast = false;
                 }
-                if (fast)
+                if (grid_kind == GRID_FP4)
+                    e = E == 64 ? launch_stream_fp4<64>(g, threads, smem2, st, a, total, exchange)
+                                : launch_stream_fp4<32>(g, threads, smem2, st, a, total, exchange);
+                else if (fast)
                     e = E == 64 ? launch_stream<64, true>(cb, g, threads, smem2, st, a, total, exchange)
                                 : launch_stream<32, true>(cb, g, threads, smem2, st, a, total, exchange);
                 else
