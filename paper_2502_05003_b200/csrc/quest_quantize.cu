@@ -187,7 +187,8 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // applied by the caller), RMS, projection, trust test, packing and stores for the E elements this
 // thread holds.  GFULL: had_block >= E, so every in-register stage runs.  FAST: the common case
 // fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
-// one warp, every output requested, no row sums -- so that no per-row branch or loop remains.
+// one warp, every output requested, no row sums, trust_factor >= 1 -- so that no per-row branch or
+// loop remains.
 template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
@@ -350,8 +351,15 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 tc.x = fminf(fmaxf(t.x, 0.0f), top);
                 tc.y = fminf(fmaxf(t.y, 0.0f), top);
                 const float2 km = __fadd2_rn(tc, magic2);
-                const float2 kf = __fadd2_rn(km, nmagic2);
-                const float2 d = __ffma2_rn(kf, neg1, t);                      // t - kf
+                float2 d;
+                if constexpr (FAST) {
+                    // trust_factor >= 1: an element inside the grid is within half a step of its level (the
+                    // difference is exact), so only clipped elements can fail, and for those level = tc
+                    d = __ffma2_rn(tc, neg1, t);                                // t - clamp(t)
+                } else {
+                    const float2 kf = __fadd2_rn(km, nmagic2);
+                    d = __ffma2_rn(kf, neg1, t);                                // t - level
+                }
                 const float dy = __fsub_rn(hh, fabsf(d.y));                    // >= +0  <=>  trusted
                 const float dx = __fsub_rn(hh, fabsf(d.x));
                 mbits = __funnelshift_l(__float_as_uint(dy), mbits, 1);         // sign bit: 1 = masked
@@ -688,7 +696,7 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 const int per_sm = smem2 > 100 * 1024 ? 1 : (E == 64 ? 2 : 4);
                 const int total = nb[0] + nb[1];
                 const int g = total < sms * per_sm ? total : sms * per_sm;
-                bool fast = had_block == 128 && S >= 32 && bits < 8;
+                bool fast = had_block == 128 && S >= 32 && bits < 8 && trust_factor >= 1.0f;
                 for (int j = 0; j < 2; ++j) {
                     const QuantTensor &t = a.t[j];
                     if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum)) fast = false;
