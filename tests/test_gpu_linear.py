@@ -118,3 +118,25 @@ def test_linear_fwd_replays_from_a_cuda_graph():
         for k in saved:
             assert torch.equal(saved[k], ref[k]), k
     assert quest.quest_device_status() == 0
+
+
+def test_two_streams_share_no_hidden_state():
+    """Calls on different streams with their own workspaces may overlap on the GPU: the library keeps
+    no mutable state between calls (apart from the timeout word), so both results equal the serial ones."""
+    import paper_2502_05003_b200 as quest
+    rng = np.random.default_rng(11)
+    xs = [to_dev(synth.f32_to_bf16_bits(rng.standard_normal((1024, 1024)).astype(np.float32))) for _ in range(2)]
+    ws = [to_dev(synth.f32_to_bf16_bits((rng.standard_normal((768, 1024)) * 0.02).astype(np.float32))) for _ in range(2)]
+    serial = [quest.quest_linear_fwd(xs[i], ws[i], 4, 128, 1.0, out_dtype=torch.bfloat16) for i in range(2)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    outs = [None, None]
+    for rep in range(5):
+        for i in range(2):
+            with torch.cuda.stream(streams[i]):
+                outs[i] = quest.quest_linear_fwd(xs[i], ws[i], 4, 128, 1.0, out_dtype=torch.bfloat16)
+        torch.cuda.synchronize()
+        for i in range(2):
+            for k in ("y", "xq", "mx", "wq", "mw", "sx", "sw"):
+                assert torch.equal(outs[i][k], serial[i][k]), (rep, i, k)
+    assert quest.quest_device_status() == 0
