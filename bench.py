@@ -39,11 +39,11 @@ L2_BYTES = 126 * 1024 * 1024
 NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 : dense bf16 tensor throughput (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, taken from the
-# committed ncu summary (profiles/); None until a capture exists.
-GEMM_DRAM_TRAFFIC_BYTES = 12651008          # profiles/gemm_i8_config2_full.md
-QUANT_DRAM_TRAFFIC_BYTES = 25188096         # profiles/quantize_stream_config2_full.md (x and w in one launch)
-QUANT_INSTR_PER_ELEMENT = 24.9              # thread instructions per element, same profile
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this command's
+# kernels (None when no capture of the current kernel exists).
+GEMM_DRAM_TRAFFIC_BYTES = 12652288          # low-bit GEMM, 4096 x 2048 x 2048
+QUANT_DRAM_TRAFFIC_BYTES = 25187584         # quantizer, x and w in one launch
+QUANT_INSTR_PER_ELEMENT = 24.4              # thread instructions per element, same capture
 
 
 def load_peaks():
