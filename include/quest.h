@@ -220,6 +220,33 @@ int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int
                          uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
                          void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Weight-only variant -- Section 4.5, "Weight-only quantization": the weights are quantized to bits_w
+ * bits as in Algorithm 1 (lines 3-4), the activations keep 16 bits.  The paper gives no algorithm of
+ * its own for this case; here it is Algorithm 1 with the rounding of line 2 left out:
+ *   x_h = bf16(HT(x))         every butterfly and the factor 1/sqrt(had_block) in binary32, in the
+ *                             quantizer's order, one rounding to bfloat16 (nearest even) at the end
+ *   w_q, sw, mw               exactly the outputs of quest_quantize(w, bits_w, had_block, trust_factor)
+ *   y[m][n] = sw[n] * sum_k x_h[m][k] c_w[n][k],   c_w = 2 k_w - (2^bits_w - 1)
+ * The sum runs on the tensor cores over bfloat16 operands (both exact) with binary32 accumulation in an
+ * order the hardware chooses, so y agrees with the exact sum to a few units of K * 2^-24 * sw[n] *
+ * sum_k |x_h c_w|, plus the rounding of y_dtype; x_h, w_q, sw and mw are reproducible bit for bit.
+ *
+ *   x [M x K], w [N x K]   device, QUEST_F32 or QUEST_BF16 each, row strides ldx / ldw elements,
+ *                          16-byte aligned rows; K a multiple of 32, 32 <= K <= 16384
+ *   y [M x N]              device, y_dtype, row stride ldy elements
+ *   xh                     optional device output [M x K] bfloat16, dense, 16-byte aligned
+ *   wq, sw, mw             optional device outputs as in quest_quantize
+ *   workspace              device scratch of at least quest_weight_only_workspace_bytes(M, N, K)
+ *                          bytes, 256-byte aligned; nothing is allocated by the call
+ * Errors as for quest_linear_fwd; M = 0 or N = 0 is QUEST_OK and launches nothing.
+ */
+int quest_linear_fwd_weight_only(const void *x, int x_dtype, int64_t ldx, const void *w, int w_dtype, int64_t ldw,
+                                 int64_t M, int64_t N, int64_t K, int bits_w, int had_block, float trust_factor,
+                                 void *y, int y_dtype, int64_t ldy, void *xh, uint8_t *wq, float *sw, uint8_t *mw,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+size_t quest_weight_only_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
 /* Bytes of scratch quest_lowbit_gemm / quest_linear_fwd need (0 on invalid arguments). */
 size_t quest_workspace_bytes(int64_t M, int64_t N, int64_t K, int bits_x, int bits_w);
 

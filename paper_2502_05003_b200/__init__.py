@@ -237,6 +237,49 @@ def quest_linear_bwd(dy: torch.Tensor, fwd: dict, bits: int, had_block: int, K: 
     return {"dx": dx, "dw": dw}
 
 
+# ---- weight-only variant (Section 4.5): b-bit weights, bfloat16 activations -----------------------
+
+def quest_weight_only_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(_lib.load().quest_weight_only_workspace_bytes(M, N, K))
+
+
+def quest_linear_fwd_weight_only(x: torch.Tensor, w: torch.Tensor, bits_w: int, had_block: int,
+                                 trust_factor: float = 1.0, out_dtype=torch.bfloat16, out: dict = None,
+                                 workspace: torch.Tensor = None) -> dict:
+    """y = HT(x) (kept in bfloat16) times the quantized w.  Returns {"y", "xh", "wq", "sw", "mw"};
+    ``out`` may hold preallocated tensors under those keys."""
+    _require_cuda(x, w, workspace)
+    if x.dim() != 2 or w.dim() != 2 or x.stride(1) != 1 or w.stride(1) != 1 or x.shape[1] != w.shape[1]:
+        raise ValueError("quest_linear_fwd_weight_only: x [M, K] and w [N, K] with unit inner stride")
+    M, K = x.shape
+    N = w.shape[0]
+    out = dict(out) if out else {}
+    cb = container_bits(bits_w)
+
+    def need(key, shape, dtype):
+        if out.get(key) is None:
+            out[key] = torch.empty(shape, dtype=dtype, device=x.device)
+        return out[key]
+
+    y = need("y", (M, N), out_dtype)
+    xh = need("xh", (M, K), torch.bfloat16)
+    wq = need("wq", (N, K * cb // 8), torch.uint8)
+    sw = need("sw", (N,), torch.float32)
+    mw = need("mw", (N, K // 8), torch.uint8)
+    _require_cuda(y, xh, wq, sw, mw)
+    if workspace is None:
+        n = quest_weight_only_workspace_bytes(M, N, K)
+        if n == 0:
+            raise ValueError("quest_linear_fwd_weight_only: unsupported shape (K a multiple of 32, 32 <= K <= 16384)")
+        workspace = torch.empty(n, dtype=torch.uint8, device=x.device)
+    st = _lib.load().quest_linear_fwd_weight_only(
+        _p(x), _dtype_code(x), x.stride(0), _p(w), _dtype_code(w), w.stride(0), M, N, K, bits_w, had_block,
+        ctypes.c_float(trust_factor), _p(y), _dtype_code(y), y.stride(0), _p(xh), _p(wq), _p(sw), _p(mw),
+        _p(workspace), workspace.numel(), _stream())
+    _lib.check(st)
+    return out
+
+
 # ---- FP4 (E2M1) grid variant: same calls with the FP4 rounding grid of Section 4.4 ---------------
 
 def quest_alpha_star_fp4() -> float:

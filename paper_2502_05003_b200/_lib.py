@@ -13,6 +13,7 @@ EXPORTS = (
     "quest_status_string", "quest_last_cuda_error", "quest_stage_timing", "quest_stage_times",
     "quest_lowbit_gemm_static", "quest_linear_bwd", "quest_bwd_workspace_bytes",
     "quest_alpha_star_fp4", "quest_quantize_fp4", "quest_lowbit_gemm_fp4", "quest_linear_fwd_fp4",
+    "quest_linear_fwd_weight_only", "quest_weight_only_workspace_bytes",
 )
 
 _lib = None
@@ -53,6 +54,11 @@ def load() -> ctypes.CDLL:
     L.quest_linear_fwd_fp4.argtypes = [vp, vp, ci, i64, i64, i64, ci, cf, vp, ci, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
     L.quest_linear_bwd.restype = ci
     L.quest_linear_bwd.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
+    L.quest_linear_fwd_weight_only.restype = ci
+    L.quest_linear_fwd_weight_only.argtypes = [vp, ci, i64, vp, ci, i64, i64, i64, i64, ci, ci, cf, vp, ci, i64,
+                                               vp, vp, vp, vp, vp, sz, vp]
+    L.quest_weight_only_workspace_bytes.restype = sz
+    L.quest_weight_only_workspace_bytes.argtypes = [i64, i64, i64]
     L.quest_bwd_workspace_bytes.restype = sz
     L.quest_bwd_workspace_bytes.argtypes = [i64, i64, i64]
     L.quest_linear_fwd.restype = ci

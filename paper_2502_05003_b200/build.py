@@ -23,6 +23,7 @@ UNITS = {
     "quest_gemm.cu": [],
     "quest_static.cu": [],
     "quest_backward.cu": [],
+    "quest_weight_only.cu": [],
 }
 
 

@@ -124,8 +124,8 @@ codes_to_bf16_t_kernel(const uint8_t *__restrict__ codes, int bits, int rows, in
 // stride: partners in other warps through shared memory, partners in this warp through shuffles,
 // the rest in registers.  A row of T = cols/32 threads occupies S slots as in the quantizer.
 __global__ void __launch_bounds__(512)
-iht_rows_kernel(const float *__restrict__ d, long long rows, int cols, int had_block, float inv_sqrt_g,
-                void *__restrict__ out, int out_dtype, long long ld, int S, int R) {
+iht_rows_kernel(const void *__restrict__ d, int in_dtype, long long ld_in, long long rows, int cols, int had_block,
+                float inv_sqrt_g, void *__restrict__ out, int out_dtype, long long ld, int S, int R) {
     extern __shared__ float xsm[];                 // [32][blockDim.x] exchange
     pdl_launch_dependents();
     pdl_wait();
@@ -135,12 +135,24 @@ iht_rows_kernel(const float *__restrict__ d, long long rows, int cols, int had_b
     const long long row = (long long)blockIdx.x * R + r_local;
     const bool active = row < rows && tr < cols / 32;
     float v[32];
-    if (active) {
-        const float4 *src = reinterpret_cast<const float4 *>(d + row * cols + (long long)tr * 32);
+    if (active && in_dtype == QUEST_F32) {
+        const float4 *src = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(d) + row * ld_in + (long long)tr * 32);
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             const float4 w = __ldg(src + q);
             v[4 * q] = w.x; v[4 * q + 1] = w.y; v[4 * q + 2] = w.z; v[4 * q + 3] = w.w;
+        }
+    } else if (active) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(d) + row * ld_in + (long long)tr * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint4 w = __ldg(src + q);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                v[8 * q + 2 * j] = __uint_as_float(ww[j] << 16);
+                v[8 * q + 2 * j + 1] = __uint_as_float(ww[j] & 0xFFFF0000u);
+            }
         }
     } else {
 #pragma unroll
@@ -223,6 +235,15 @@ BwdWorkspace carve_bwd(void *base, int64_t M, int64_t N, int64_t K) {
 
 int launch_iht(const float *d, int64_t rows, int64_t cols, int had_block, void *out, int out_dtype, int64_t ld,
                cudaStream_t st) {
+    return launch_hadamard_rows(d, QUEST_F32, cols, rows, cols, had_block, out, out_dtype, ld, st);
+}
+
+}  // namespace
+
+// Orthonormal block Hadamard transform (its own inverse) of every row: in [rows x cols] with row
+// stride ld_in (16-byte aligned rows), out with row stride ld; cols % 32 == 0.
+int launch_hadamard_rows(const void *in, int in_dtype, int64_t ld_in, int64_t rows, int64_t cols, int had_block,
+                         void *out, int out_dtype, int64_t ld, cudaStream_t st) {
     if (rows == 0) return QUEST_OK;
     const int T = (int)(cols / 32);
     int S;
@@ -235,10 +256,13 @@ int launch_iht(const float *d, int64_t rows, int64_t cols, int had_block, void *
         if (e != cudaSuccess) return cuda_fail(e);
     }
     const long long grid = (rows + R - 1) / R;
-    cudaError_t e = launch_pdl(iht_rows_kernel, dim3((unsigned)grid), dim3(threads), smem, st, 1, d, (long long)rows, (int)cols,
-                               had_block, 1.0f / sqrtf((float)had_block), out, out_dtype, (long long)ld, S, R);
+    cudaError_t e = launch_pdl(iht_rows_kernel, dim3((unsigned)grid), dim3(threads), smem, st, 1, in, in_dtype, (long long)ld_in,
+                               (long long)rows, (int)cols, had_block, 1.0f / sqrtf((float)had_block), out, out_dtype,
+                               (long long)ld, S, R);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
+
+namespace {
 
 bool bwd_shape_ok(int64_t M, int64_t N, int64_t K) {
     return M > 0 && N > 0 && K >= 32 && K % 32 == 0 && K <= 16384 && M % 8 == 0 && N % 8 == 0 &&

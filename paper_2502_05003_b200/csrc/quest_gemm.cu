@@ -249,14 +249,17 @@ struct SmemLayout {
 // codes.  MODE 2 (backward pass, Algorithm 2): bfloat16 operands (kind::f16, binary32 accumulators);
 // the epilogue zeroes the elements the trust mask rejects and stores binary32.  MODE 3: MODE 2 plus
 // the inverse Hadamard transform for blocks of 128 fused into the epilogue (BN = 256: the 128
-// columns a thread holds are exactly one block), output in the caller's type.
+// columns a thread holds are exactly one block), output in the caller's type.  MODE 4 (weight-only
+// variant): bfloat16 operands, y = sw[n] * accumulator.
 template <int BN, int MODE, bool TWO, bool YT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
     using L = SmemLayout<BN, TWO>;
     constexpr bool CORR = MODE == 1;
-    constexpr bool BWD = MODE >= 2;
+    constexpr bool BWD = MODE == 2 || MODE == 3;
+    constexpr bool F16 = MODE >= 2;               // bfloat16 operands, binary32 accumulators
+    constexpr bool WO = MODE == 4;
     constexpr bool IHT128 = MODE == 3;
     static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
     constexpr int STAGES = L::NSTAGES;
@@ -360,7 +363,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0 && leader) {
-            constexpr uint32_t idesc = BWD ? make_idesc_bf16(TILE_M, BN) : make_idesc_i8(TILE_M, BN);
+            constexpr uint32_t idesc = F16 ? make_idesc_bf16(TILE_M, BN) : make_idesc_i8(TILE_M, BN);
             int stage = 0;
             uint32_t phase = 0;
             int t = 0;
@@ -385,7 +388,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const uint64_t ad = a_desc + (uint64_t)(kk * (UMMA_K >> 4));
                         const uint64_t bd = b_desc + (uint64_t)(kk * (UMMA_K >> 4));
                         const uint32_t accum = (kb | kk) != 0 ? 1u : 0u;
-                        if constexpr (BWD) {      // 32 bytes of K = 16 bfloat16 per instruction
+                        if constexpr (F16) {      // 32 bytes of K = 16 bfloat16 per instruction
                             if constexpr (TWO) umma_bf16_pair(d_tmem, ad, bd, idesc, accum);
                             else umma_bf16(d_tmem, ad, bd, idesc, accum);
                         } else {
@@ -440,7 +443,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // without 8-bit corrections and without the raw accumulators, the exact power of two of the
             // operand scaling is folded into the row scale instead of shifting every accumulator
             const bool fold = !CORR && !p.acc;
-            float sxr = (!BWD && row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
+            float sxr = WO ? 1.0f : (!BWD && row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
             if (fold) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.sh) << 23));
             if (p.ysh) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.ysh) << 23));
             int rsa = 0;
@@ -552,7 +555,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const float2 *sw2 = reinterpret_cast<const float2 *>(swt + cbase + c0);
 #pragma unroll
                         for (int j = 0; j < (BWD ? 0 : 32); j += 2) {
-                            const float2 a2 = make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
+                            const float2 a2 = WO ? make_float2(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]))
+                                                 : make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
                             const float2 y2 = __fmul2_rn(__fmul2_rn(sx2, sw2[j >> 1]), a2);
                             rc[j] = __float_as_uint(y2.x);
                             rc[j + 1] = __float_as_uint(y2.y);
@@ -931,6 +935,38 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     if (pair) return launch_gemm_bn<256, 2, true, true>(tmA, tmB, tmY, p, st);
     if (wide) return launch_gemm_bn<256, 2, false, true>(tmA, tmB, tmY, p, st);
     return launch_gemm_bn<128, 2, false, true>(tmA, tmB, tmY, p, st);
+}
+
+int launch_gemm_bf16_scaled(const void *a, const void *b, const float *sw, int64_t M, int64_t N, int64_t K,
+                            void *y, int y_dtype, int64_t ldy, cudaStream_t st) {
+    if (M == 0 || N == 0) return QUEST_OK;
+    GemmParams p;
+    p.M = (int)M; p.N = (int)N; p.K = (int)(2 * K);
+    p.sx = nullptr; p.sw = sw; p.rs_a = nullptr; p.rs_b = nullptr;
+    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; p.ysh = 0;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = nullptr; p.mask = nullptr;
+    p.status = device_status_word();
+    if (!p.status) return QUEST_ERR_CUDA;
+    const bool wide = N > 128;
+    const bool pair = wide && M > 128;
+    CUtensorMap tmA, tmB;
+    int s = make_operand_map(&tmA, reinterpret_cast<const int8_t *>(a), M, 2 * K, BM);
+    if (s) return s;
+    s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(b), N, 2 * K, pair ? 128 : wide ? 256 : 128);
+    if (s) return s;
+    const size_t esz = y_dtype == QUEST_F32 ? 4 : 2;
+    const bool yt = (reinterpret_cast<uintptr_t>(y) % 16 == 0) && ((size_t)ldy * esz % 16 == 0);
+    CUtensorMap tmY = tmA;
+    if (yt) {
+        s = make_output_map(&tmY, y, M, (int64_t)N * (int64_t)esz, (int64_t)ldy * (int64_t)esz);
+        if (s) return s;
+    }
+#define QUEST_GEMM_WO(BNV, TWOV) \
+    (yt ? launch_gemm_bn<BNV, 4, TWOV, true>(tmA, tmB, tmY, p, st) : launch_gemm_bn<BNV, 4, TWOV, false>(tmA, tmB, tmY, p, st))
+    if (pair) return QUEST_GEMM_WO(256, true);
+    if (wide) return QUEST_GEMM_WO(256, false);
+    return QUEST_GEMM_WO(128, false);
+#undef QUEST_GEMM_WO
 }
 
 }  // namespace quest
