@@ -109,6 +109,8 @@ struct QuantJob {
     uint8_t *mask;
     int8_t *op8;
     int32_t *rowsum;
+    uint16_t *rot = nullptr;   // [rows x cols] bfloat16 of the orthonormal rotation (no quantization needed for it)
+    uint16_t *cbf = nullptr;   // [rows x cols] grid values as bfloat16
 };
 // Up to two tensors with the same row length, dtype and parameters share one launch.
 int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
@@ -131,8 +133,6 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
 // Orthonormal block Hadamard transform of every row (binary32 or bfloat16 in, binary32 or bfloat16 out).
 int launch_hadamard_rows(const void *in, int in_dtype, int64_t ld_in, int64_t rows, int64_t cols, int had_block,
                          void *out, int out_dtype, int64_t ld, cudaStream_t st);
-// Packed level indices -> grid values c = 2k - (2^b - 1) as bfloat16 (exact), dense [rows x K].
-int launch_codes_to_bf16(const uint8_t *codes, int bits, int64_t rows, int64_t K, void *out, cudaStream_t st);
 // Weight-only contraction: y[m][n] = sw[n] * sum_k a[m][k] b[n][k], bfloat16 operands (dense, K contiguous),
 // binary32 accumulation.
 int launch_gemm_bf16_scaled(const void *a, const void *b, const float *sw, int64_t M, int64_t N, int64_t K,

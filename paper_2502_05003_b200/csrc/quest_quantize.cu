@@ -8,6 +8,8 @@
 // inv = A/rms; t = fma(u, inv, c0); level = rint(clamp(t, 0, 2^b-1)) (ties to even);
 // trusted = |t - level| <= trust_factor/2.  This file is compiled with -fmad=false and uses
 // the explicit _rn intrinsics so that the compiler cannot fuse or reorder any of it.
+#include <cuda_bf16.h>
+
 #include "quest_internal.cuh"
 #include "quest_operand.cuh"
 
@@ -158,12 +160,15 @@ struct QuantTensor {
     uint8_t *mask;
     int8_t *op8;
     int32_t *rowsum;       // sum of the row's operand bytes (needed by the GEMM for 8-bit codes)
+    uint16_t *rot;         // bfloat16 of the orthonormal rotation itself (weight-only variant)
+    uint16_t *cbf;         // grid values c = 2k - (2^b - 1) as bfloat16 (weight-only variant)
 };
 struct QuantArgs {
     QuantTensor t[2];
     int blocks0;
     int cols, bits, had_block;
     QuantConsts qc;
+    float inv_sqrt_g;      // 1 / sqrt(had_block) in binary32
     int S, R;
 };
 
@@ -262,6 +267,28 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
         for (int i = 0; i < H; ++i) {
             const float p = v[i].x, q = v[i].y;
             v[i] = make_float2(__fadd_rn(p, q), __fsub_rn(p, q));
+        }
+    }
+
+    // ---- the rotation itself as an output (weight-only variant): x_h = bf16(u / sqrt(g)) -----
+    if constexpr (!FAST) {
+        if (tn.rot) {                                           // uniform over the CTA
+            if (active) {
+                const float2 ig = make_float2(a.inv_sqrt_g, a.inv_sqrt_g);
+                uint4 *dst = reinterpret_cast<uint4 *>(tn.rot + row * (long long)cols + (long long)tr * E);
+#pragma unroll
+                for (int q = 0; q < E / 8; ++q) {
+                    uint32_t o[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 p = __fmul2_rn(v[q * 4 + j], ig);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(p.x, p.y);
+                        o[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    dst[q] = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+            if (!tn.codes && !tn.scales && !tn.mask && !tn.op8 && !tn.rowsum && !tn.cbf) return;   // nothing else asked for
         }
     }
 
@@ -397,6 +424,26 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                     reinterpret_cast<uint2 *>(dst)[0] = make_uint2(w[0], w[1]);
                 } else {
                     reinterpret_cast<uint32_t *>(dst)[0] = w[0];
+                }
+            }
+            if constexpr (!FAST && GRID == GRID_UNIFORM) {
+                if (tn.cbf) {
+                    // a small integer as bfloat16 is the upper half of its binary32 pattern (|c| <= 255: exact)
+                    const int L1 = (1 << a.bits) - 1;
+                    uint4 *dst = reinterpret_cast<uint4 *>(tn.cbf + row * (long long)cols + (long long)tr * E + g32 * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int e0 = 8 * q + 2 * j, e1 = e0 + 1;
+                            const int k0 = (int)((w[e0 / PER] >> ((e0 % PER) * CB)) & ((1u << CB) - 1u));
+                            const int k1 = (int)((w[e1 / PER] >> ((e1 % PER) * CB)) & ((1u << CB) - 1u));
+                            o[j] = (__float_as_uint((float)(2 * k0 - L1)) >> 16) |
+                                   (__float_as_uint((float)(2 * k1 - L1)) & 0xFFFF0000u);
+                        }
+                        dst[q] = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
                 }
             }
             if (FAST || tn.op8) {
@@ -666,16 +713,17 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 if (j0 + j < njobs) {
                     const QuantJob &q = jobs[j0 + j];
                     t.x = q.x; t.rows = q.rows; t.ld = q.ld; t.codes = q.codes; t.scales = q.scales;
-                    t.mask = q.mask; t.op8 = q.op8; t.rowsum = q.rowsum;
+                    t.mask = q.mask; t.op8 = q.op8; t.rowsum = q.rowsum; t.rot = q.rot; t.cbf = q.cbf;
                     nb[j] = (int)((q.rows + R - 1) / R);
                 } else {
                     t.x = nullptr; t.rows = 0; t.ld = 0; t.codes = nullptr; t.scales = nullptr;
-                    t.mask = nullptr; t.op8 = nullptr; t.rowsum = nullptr;
+                    t.mask = nullptr; t.op8 = nullptr; t.rowsum = nullptr; t.rot = nullptr; t.cbf = nullptr;
                 }
             }
             if (nb[0] + nb[1] == 0) continue;
             a.blocks0 = nb[0];
             a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = S; a.R = R;
+            a.inv_sqrt_g = 1.0f / sqrtf((float)had_block);
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
             const bool streaming = (E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64;
@@ -699,7 +747,7 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 bool fast = had_block == 128 && S >= 32 && bits < 8 && trust_factor >= 1.0f;
                 for (int j = 0; j < 2; ++j) {
                     const QuantTensor &t = a.t[j];
-                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum)) fast = false;
+                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum && !t.rot && !t.cbf)) fast = false;
                 }
                 if (grid_kind == GRID_FP4)
                     e = E == 64 ? launch_stream_fp4<64>(g, threads, smem2, st, a, total, exchange)

@@ -2,9 +2,9 @@
 // rounding of the activations left out.  The weights go through the full quantizer; the
 // activations are rotated by the same block Hadamard transform and stay in bfloat16:
 //
-//   x_h = bf16(HT(x))                     launch_hadamard_rows  (binary32 butterflies, one rounding)
-//   w -> codes, sw, trust mask            launch_quantize
-//   c_w = bf16(2k - (2^b - 1))            codes_to_bf16_kernel  (exact: |c| <= 255)
+//   x_h = bf16(HT(x))                     quantizer launch, rotation output (binary32 butterflies, one rounding)
+//   w -> codes, sw, trust mask,           same launch
+//        c_w = bf16(2k - (2^b - 1))       (exact: |c| <= 255)
 //   y[m][n] = sw[n] sum_k x_h[m][k] c_w[n][k]    tcgen05 kind::f16 contraction, binary32 accumulators
 #include <cuda_bf16.h>
 
@@ -12,36 +12,6 @@
 
 namespace quest {
 namespace {
-
-// One thread converts 32 consecutive elements of a row (rows are dense, K % 32 == 0).
-template <int CB>
-__global__ void __launch_bounds__(256)
-codes_to_bf16_kernel(const uint8_t *__restrict__ codes, int bits, long long n_groups, uint16_t *__restrict__ out) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const long long gidx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (gidx >= n_groups) return;
-    constexpr int PER = 32 / CB;
-    const int L1 = (1 << bits) - 1;
-    uint32_t w[CB];
-    const uint32_t *src = reinterpret_cast<const uint32_t *>(codes) + gidx * CB;
-#pragma unroll
-    for (int q = 0; q < CB; ++q) w[q] = __ldg(src + q);
-    uint4 *dst = reinterpret_cast<uint4 *>(out + gidx * 32);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {                       // 8 elements per 16-byte store
-        uint32_t o[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int e0 = 8 * q + 2 * j, e1 = e0 + 1;
-            const int k0 = (w[e0 / PER] >> ((e0 % PER) * CB)) & ((1 << CB) - 1);
-            const int k1 = (w[e1 / PER] >> ((e1 % PER) * CB)) & ((1 << CB) - 1);
-            // a small integer as bfloat16: the upper half of its binary32 pattern (no rounding: |c| <= 255)
-            o[j] = (__float_as_uint((float)(2 * k0 - L1)) >> 16) | (__float_as_uint((float)(2 * k1 - L1)) & 0xFFFF0000u);
-        }
-        dst[q] = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-}
 
 struct WoWorkspace {
     uint16_t *xh;      // [M x K] rotated activations
@@ -68,21 +38,6 @@ bool wo_shape_ok(int64_t M, int64_t N, int64_t K) {
 }
 
 }  // namespace
-
-int launch_codes_to_bf16(const uint8_t *codes, int bits, int64_t rows, int64_t K, void *out, cudaStream_t st) {
-    const long long n_groups = (long long)rows * (K / 32);
-    if (n_groups == 0) return QUEST_OK;
-    const dim3 grid((unsigned)((n_groups + 255) / 256));
-    uint16_t *o = reinterpret_cast<uint16_t *>(out);
-    cudaError_t e;
-    switch (container_bits(bits)) {
-        case 1: e = launch_pdl(codes_to_bf16_kernel<1>, grid, dim3(256), 0, st, 1, codes, bits, n_groups, o); break;
-        case 2: e = launch_pdl(codes_to_bf16_kernel<2>, grid, dim3(256), 0, st, 1, codes, bits, n_groups, o); break;
-        case 4: e = launch_pdl(codes_to_bf16_kernel<4>, grid, dim3(256), 0, st, 1, codes, bits, n_groups, o); break;
-        default: e = launch_pdl(codes_to_bf16_kernel<8>, grid, dim3(256), 0, st, 1, codes, bits, n_groups, o); break;
-    }
-    return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
-}
 
 }  // namespace quest
 
@@ -122,16 +77,18 @@ extern "C" int quest_linear_fwd_weight_only(const void *x, int x_dtype, int64_t 
     uint8_t *wq_buf = wq ? wq : ws.wq;
     float *sw_buf = sw ? sw : ws.sw;
     {
+        // one launch when x and w share a type: rows of x leave as x_h, rows of w as codes, scale, mask and
+        // bfloat16 grid values
         void *h = stage_begin(QUEST_STAGE_QUANT_W, st);
-        QuantJob job = {w, N, ldw, wq_buf, sw_buf, mw, nullptr, nullptr};
-        s = launch_quantize(&job, 1, w_dtype, K, bits_w, had_block, trust_factor, st);
-        stage_end(h);
-        if (s) return s;
-    }
-    {
-        void *h = stage_begin(QUEST_STAGE_UNPACK, st);
-        s = launch_hadamard_rows(x, x_dtype, ldx, M, K, had_block, xh_buf, QUEST_BF16, K, st);
-        if (!s) s = launch_codes_to_bf16(wq_buf, bits_w, N, K, ws.cw, st);
+        QuantJob jobs[2];
+        jobs[0] = QuantJob{x, M, ldx, nullptr, nullptr, nullptr, nullptr, nullptr, xh_buf, nullptr};
+        jobs[1] = QuantJob{w, N, ldw, wq_buf, sw_buf, mw, nullptr, nullptr, nullptr, ws.cw};
+        if (x_dtype == w_dtype) {
+            s = launch_quantize(jobs, 2, x_dtype, K, bits_w, had_block, trust_factor, st);
+        } else {
+            s = launch_quantize(&jobs[0], 1, x_dtype, K, bits_w, had_block, trust_factor, st);
+            if (!s) s = launch_quantize(&jobs[1], 1, w_dtype, K, bits_w, had_block, trust_factor, st);
+        }
         stage_end(h);
         if (s) return s;
     }
