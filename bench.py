@@ -2,7 +2,7 @@
 """Benchmark of the QuEST quantized-linear forward hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--had-block G]
-                    [--no-graph] [--pass backward]
+                    [--no-graph] [--pass backward|weight_only]
 
 One "step" is one pass of the whole path (Algorithm 1: quantize X, quantize W, low-bit GEMM with
 the dequantising epilogue) through the C ABI call ``quest_linear_fwd`` on the 1.6B-scale layer:
@@ -10,7 +10,8 @@ X[4096 x 2048] bf16, W[2048 x 2048] bf16, b = 4, Hadamard block 128 (seeded synt
 The step rotates over a ring of buffer sets larger than L2, so every step streams from HBM, and the
 timed steps are replayed from a CUDA graph holding one pass over the ring (``--no-graph``: direct
 launches), because the host cannot launch a step of a few tens of microseconds fast enough.
-``--pass backward`` times Algorithm 2 (``quest_linear_bwd``) on the same layer instead.
+``--pass backward`` times Algorithm 2 (``quest_linear_bwd``) on the same layer instead, and
+``--pass weight_only`` the weight-only forward of Section 4.5 (``quest_linear_fwd_weight_only``).
 
 Prints ONE JSON line (rank 0).  ``value`` is tokens/s with inputs resident in HBM; ``e2e`` is the
 same metric with the host->device copy of X and W and the device->host copy of y inside the
@@ -578,6 +579,124 @@ def run_backward(args, rank: int, world: int, local: int):
     print(json.dumps(line), flush=True)
 
 
+def run_weight_only(args, rank: int, world: int, local: int):
+    """Weight-only variant (Section 4.5) on the same layer: `python bench.py --pass weight_only`.  One step =
+    quest_linear_fwd_weight_only (W4, bfloat16 activations); same ring / graph / event method."""
+    import numpy as np
+    import torch
+
+    import paper_2502_05003_b200 as quest
+    from paper_2502_05003_b200 import synth
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    g = args.had_block
+    cfg = synth.config2()
+    M, K, N = TOKENS, HIDDEN, OUT
+    x_host = torch.from_numpy(cfg["x"]).view(torch.bfloat16)
+    w_host = torch.from_numpy(cfg["w"]).view(torch.bfloat16)
+    ws_bytes = quest.quest_weight_only_workspace_bytes(M, N, K)
+
+    def make_set():
+        return {"x": x_host.to(dev), "w": w_host.to(dev),
+                "out": {"y": torch.empty((M, N), dtype=torch.bfloat16, device=dev),
+                        "xh": torch.empty((M, K), dtype=torch.bfloat16, device=dev),
+                        "wq": torch.empty((N, K // 2), dtype=torch.uint8, device=dev),
+                        "sw": torch.empty(N, dtype=torch.float32, device=dev),
+                        "mw": torch.empty((N, K // 8), dtype=torch.uint8, device=dev)},
+                "ws": torch.empty(ws_bytes, dtype=torch.uint8, device=dev)}
+
+    set_bytes = (M + N) * K * 2 + M * K * 2 + N * K * (0.5 + 0.125 + 2) + M * N * 2
+    n_sets = max(2, int(np.ceil(3.0 * L2_BYTES / set_bytes)))
+    ring = [make_set() for _ in range(n_sets)]
+
+    def step(i):
+        s = ring[i % n_sets]
+        quest.quest_linear_fwd_weight_only(s["x"], s["w"], BITS, g, 1.0, out=s["out"], workspace=s["ws"])
+
+    def capture():
+        if args.no_graph:
+            return None
+        side = torch.cuda.Stream(device=dev)
+        g_ = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            for i in range(n_sets):
+                step(i)
+            side.synchronize()
+            with torch.cuda.graph(g_, stream=side):
+                for i in range(n_sets):
+                    step(i)
+        torch.cuda.synchronize()
+        return g_
+
+    def run_steps(k, graph):
+        if graph is None:
+            for i in range(k):
+                step(i)
+            return
+        for _ in range(k // n_sets):
+            graph.replay()
+        for i in range(k % n_sets):
+            step(i)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    graph = capture()
+    run_steps(n_sets, graph)
+    torch.cuda.synchronize()
+    steps = min(args.steps, 500)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        run_steps(steps, graph)
+        e1.record()
+        torch.cuda.synchronize()
+    elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3, world, dev)
+    if quest.quest_device_status() != 0:
+        raise RuntimeError("device status after the timed region")
+    quest.quest_stage_timing(True)
+    quest.quest_stage_times(reset=2)
+    staged = capture()
+    for r in range(30):
+        if staged is None:
+            step(r)
+        else:
+            staged.replay()
+        quest.quest_stage_times()
+    stage = quest.quest_stage_times(reset=2)
+    quest.quest_stage_timing(False)
+    stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+    if rank != 0:
+        return
+    peaks = load_peaks()
+    gemm_ms = stage_ms["gemm"]
+    tflops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12 if gemm_ms else None
+    from oracle import weight_only as wo
+    sample = 256
+    t0 = time.perf_counter()
+    wo.linear_fwd_weight_only(cfg["x"][:sample], cfg["w"], BITS, g, 1.0)
+    o_dt = time.perf_counter() - t0
+    line = {
+        "metric": "QuEST W4A16 (weight-only) linear fwd tokens/s", "value": M * steps * world / elapsed, "unit": UNIT,
+        "n_gpus": world, "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * elapsed / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": dict(workload_config(g), workload="config 2, weight-only: X[4096x2048] bf16 x W4[2048x2048] -> y bf16",
+                       l2="ring of %d buffer sets (%.0f MB) larger than L2" % (n_sets, n_sets * set_bytes / 1e6)),
+        "gpu_launches": 2 * steps, "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
+        "clocks": clocks.summary(),
+        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel<mode 4> (tcgen05 kind::f16 bf16, column-scale epilogue)",
+                     "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": (tflops / peaks["bf16_tflops"]) if tflops else None,
+                     "peak_basis": "bf16 burst " + ("of measured" if peaks["_source"] == "measured" else "of fallback"),
+                     "traffic": None, "ms": gemm_ms},
+        "stage_ms": {"rotate_and_quantize": stage_ms["quant_w"], "gemm": gemm_ms},
+        "cpu_baseline": {"value": sample / o_dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                         "sample": "%d of %d token rows against the full W (weights quantized in full)" % (sample, M)},
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -586,8 +705,9 @@ def main():
     ap.add_argument("--impl", default="quest", choices=["quest", "reference"])
     ap.add_argument("--had-block", type=int, default=128)
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
-    ap.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward"],
-                    help="forward: Algorithm 1, the headline metric (default); backward: Algorithm 2 on the same layer")
+    ap.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward", "weight_only"],
+                    help="forward: Algorithm 1, the headline metric (default); backward: Algorithm 2 on the same layer; "
+                         "weight_only: the W4A16 forward of Section 4.5 on the same layer")
     ap.add_argument("--ref-tokens", type=int, default=0,
                     help="token rows in the CPU oracle's bounded sample (0: the full 4096 for the "
                          "cpu_baseline leg; sized to about a minute in total for --impl reference)")
@@ -598,6 +718,9 @@ def main():
         return
     if args.which == "backward":
         run_backward(args, rank, world, local)
+        return
+    if args.which == "weight_only":
+        run_weight_only(args, rank, world, local)
         return
     run_gpu(args, rank, world, local)
 
