@@ -200,10 +200,13 @@ size_t quest_bwd_workspace_bytes(int64_t M, int64_t N, int64_t K);
  * trust_factor).  Formats: codes are E2M1 nibbles (sign << 3 | magnitude index, two per byte,
  * element 0 in the low nibble, rounded to nearest even and saturated by the hardware conversion);
  * scale[row] = alpha*_FP4 RMS(x_h) / 6, so the dequantised element is scale * E2M1 value; masks as for
- * the uniform grid.  The contraction runs on the int8 tensor cores with operands 2 v (exact):
- * acc4[i][j] = 4 sum_k v_x v_w in int32, y = sx[i] sw[j] acc4 / 4.
+ * the uniform grid.  The contraction runs on the FP4 tensor-core path (tcgen05 kind::mxf4 with every
+ * block scale 2^0) directly on the packed codes; its binary32 accumulators hold sum_k v_x v_w exactly
+ * (multiples of 1/4 below 2^22 for every supported K), reported as acc4[i][j] = 4 sum_k v_x v_w in int32,
+ * and y = sx[i] sw[j] acc4 / 4.
  * Arguments and rules are those of quest_quantize / quest_lowbit_gemm / quest_linear_fwd with
- * bits = 4; cols (K) must be a multiple of 32.
+ * bits = 4; cols (K) must be a multiple of 32 and xq, wq 16-byte aligned.  Nothing is unpacked, so
+ * the workspace arguments of the two GEMM-bearing calls are unused and may be NULL / 0.
  */
 float quest_alpha_star_fp4(void);
 int quest_quantize_fp4(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld_elems,

@@ -306,10 +306,10 @@ def quest_lowbit_gemm_fp4(xq, sx, wq, sw, K: int, out_dtype=torch.bfloat16, want
     M, N = xq.shape[0], wq.shape[0]
     y = torch.empty((M, N), dtype=out_dtype, device=xq.device)
     acc = torch.empty((M, N), dtype=torch.int32, device=xq.device) if want_acc else None
-    if workspace is None:
-        workspace = alloc_workspace(M, N, K, 4, 4, xq.device)
+    # the packed codes are the tensor-core operands: the call needs no scratch (the argument is kept in the ABI)
     _lib.check(_lib.load().quest_lowbit_gemm_fp4(_p(xq), _p(sx), _p(wq), _p(sw), M, N, K, _p(y), _dtype_code(y),
-                                                 y.stride(0), _p(acc), _p(workspace), workspace.numel(), _stream()))
+                                                 y.stride(0), _p(acc), _p(workspace),
+                                                 workspace.numel() if workspace is not None else 0, _stream()))
     return y, acc
 
 
@@ -332,11 +332,9 @@ def quest_linear_fwd_fp4(x: torch.Tensor, w: torch.Tensor, had_block: int, trust
     out["sx"] = torch.empty(M, dtype=torch.float32, device=dev)
     out["mx"] = torch.empty((M, K // 8), dtype=torch.uint8, device=dev)
     y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=dev)
-    if workspace is None:
-        workspace = alloc_workspace(M, N, K, 4, 4, dev)
     _lib.check(_lib.load().quest_linear_fwd_fp4(
         _p(x), _p(w), _dtype_code(x), M, N, K, had_block, ctypes.c_float(trust_factor), _p(y), _dtype_code(y),
         _p(out["xq"]), _p(out["sx"]), _p(out["mx"]), _p(out["wq"]), _p(out["sw"]), _p(out["mw"]),
-        1 if w_cached is not None else 0, _p(workspace), workspace.numel(), _stream()))
+        1 if w_cached is not None else 0, _p(workspace), workspace.numel() if workspace is not None else 0, _stream()))
     out["y"] = y
     return out

@@ -346,18 +346,12 @@ int quest_lowbit_gemm_fp4(const uint8_t *xq, const float *sx, const uint8_t *wq,
         if (!aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
     }
     if (!aligned(xq, 16) || !aligned(wq, 16) || (acc4 && !aligned(acc4, 4))) return QUEST_ERR_ALIGN;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, 4, 4))
-        return QUEST_ERR_WORKSPACE;
     if ((s = check_device())) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    Workspace ws = carve_workspace(workspace, M, N, K);
-    {
-        StageScope scope(QUEST_STAGE_UNPACK, st);
-        if ((s = launch_unpack(xq, 4, M, K, ws.a8, nullptr, st, GRID_FP4))) return s;
-        if ((s = launch_unpack(wq, 4, N, K, ws.b8, nullptr, st, GRID_FP4))) return s;
-    }
+    (void)workspace;
+    (void)workspace_bytes;
     StageScope scope(QUEST_STAGE_GEMM, st);
-    return launch_gemm(ws.a8, ws.b8, nullptr, nullptr, 4, 4, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc4, st, GRID_FP4);
+    return launch_gemm_mxfp4(xq, wq, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc4, st);
 }
 
 int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
@@ -373,27 +367,24 @@ int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int
     if (s) return s;
     if ((s = validate_quantize(x, dtype, M, K, K, 4, had_block, trust_factor, xq, mx))) return s;
     if (!w_is_cached && (s = validate_quantize(w, dtype, N, K, K, 4, had_block, trust_factor, wq, mw))) return s;
-    if (!aligned(wq, 16) || !aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, 4, 4))
-        return QUEST_ERR_WORKSPACE;
+    if (!aligned(xq, 16) || !aligned(wq, 16) || !aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
     if ((s = check_device())) return s;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    Workspace ws = carve_workspace(workspace, M, N, K);
-    const QuantJob jx = {x, M, K, xq, sx, mx, ws.a8, nullptr};
-    if (w_is_cached) {
-        {
-            StageScope scope(QUEST_STAGE_QUANT_X, st);
-            if ((s = launch_quantize(&jx, 1, dtype, K, 4, had_block, trust_factor, st, GRID_FP4))) return s;
-        }
-        StageScope scope(QUEST_STAGE_UNPACK, st);
-        if ((s = launch_unpack(wq, 4, N, K, ws.b8, nullptr, st, GRID_FP4))) return s;
-    } else {
+    (void)workspace;
+    (void)workspace_bytes;
+    // the packed codes are the tensor-core operands: nothing is unpacked
+    const QuantJob jx = {x, M, K, xq, sx, mx, nullptr, nullptr};
+    {
         StageScope scope(QUEST_STAGE_QUANT_X, st);
-        const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, ws.b8, nullptr}};
-        if ((s = launch_quantize(jobs, 2, dtype, K, 4, had_block, trust_factor, st, GRID_FP4))) return s;
+        if (w_is_cached) {
+            if ((s = launch_quantize(&jx, 1, dtype, K, 4, had_block, trust_factor, st, GRID_FP4))) return s;
+        } else {
+            const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, nullptr, nullptr}};
+            if ((s = launch_quantize(jobs, 2, dtype, K, 4, had_block, trust_factor, st, GRID_FP4))) return s;
+        }
     }
     StageScope scope(QUEST_STAGE_GEMM, st);
-    return launch_gemm(ws.a8, ws.b8, nullptr, nullptr, 4, 4, sx, sw, M, N, K, y, y_dtype, N, nullptr, st, GRID_FP4);
+    return launch_gemm_mxfp4(xq, wq, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);
 }
 
 }  // extern "C"

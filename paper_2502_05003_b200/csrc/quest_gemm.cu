@@ -10,6 +10,9 @@
 // for b = 8 (|c| up to 255) it is v = k - 128 and the epilogue restores
 // c_x . c_w = 4 v_x.v_w + 2 sum(v_x) + 2 sum(v_w) + K exactly from per-row sums.
 //
+// The FP4 grid (Section 4.4) has a native operand type: its packed E2M1 codes feed tcgen05.mma
+// kind::mxf4 directly (MODE 5 below), with all block scales 2^0.
+//
 // Two launch shapes of one kernel template.  TWO = false: one CTA per SM, persistent over 128 x BN
 // output tiles.  TWO = true: clusters of two CTAs (tcgen05 cta_group::2) persistent over 256 x 256
 // tiles; each CTA stages its own 128 rows of A and its own 128 of the tile's 256 rows of B, the
@@ -57,7 +60,6 @@ struct GemmParams {
     const int32_t *rs_b;   // row sums of the B operand values (nullable)
     int mul;               // acc' = (mul*acc + ca*rs_a[i] + cb*rs_b[j] + ck) >> sh   (exact)
     int ca, cb, ck, sh;
-    int ysh;               // y carries an extra exact factor 2^-ysh (FP4 grid: operands are twice the E2M1 values)
     void *y;
     int y_dtype;
     long long ldy;
@@ -150,6 +152,35 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// kind::mxf4 (Section 4.4, FP4): A and B are packed E2M1 (two per byte, K-major, 64 elements of K per
+// instruction), accumulation in binary32, one UE8M0 scale per 32 elements of K read from tensor
+// memory.  The low-bit path uses no block scales, so every scale byte is 2^0.
+__host__ __device__ constexpr uint32_t make_idesc_mxf4(int m, int n) {
+    return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate, uint32_t sfa_tmem, uint32_t sfb_tmem) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+        : "memory");
+}
+__device__ __forceinline__ void umma_mxf4_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate, uint32_t sfa_tmem, uint32_t sfb_tmem) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+        : "memory");
+}
+// Four columns of this warp's 32 tensor-memory lanes <- one word each.
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, uint32_t v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v), "r"(v), "r"(v), "r"(v)
+                 : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
@@ -250,7 +281,10 @@ struct SmemLayout {
 // the epilogue zeroes the elements the trust mask rejects and stores binary32.  MODE 3: MODE 2 plus
 // the inverse Hadamard transform for blocks of 128 fused into the epilogue (BN = 256: the 128
 // columns a thread holds are exactly one block), output in the caller's type.  MODE 4 (weight-only
-// variant): bfloat16 operands, y = sw[n] * accumulator.
+// variant): bfloat16 operands, y = sw[n] * accumulator.  MODE 5 (FP4 grid): packed E2M1 operands on
+// kind::mxf4 with unit block scales; the binary32 accumulators hold sum v_x v_w exactly (multiples of
+// 1/4 below 2^22), reported as acc4 = 4 * sum; tensor memory holds one accumulator buffer of 256
+// columns (or two of 128) and the scale bytes.
 template <int BN, int MODE, bool TWO, bool YT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -260,6 +294,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr bool BWD = MODE == 2 || MODE == 3;
     constexpr bool F16 = MODE >= 2;               // bfloat16 operands, binary32 accumulators
     constexpr bool WO = MODE == 4;
+    constexpr bool MX = MODE == 5;
+    constexpr int NBUF = (MX && BN == 256) ? 1 : 2;   // accumulator buffers in tensor memory
+    constexpr uint32_t SF_COL = 256;              // MX: 32 columns of scale bytes after the accumulators
     constexpr bool IHT128 = MODE == 3;
     static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
     constexpr int STAGES = L::NSTAGES;
@@ -278,7 +315,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    constexpr uint32_t TMEM_COLS = 2 * BN;       // two accumulator buffers
+    constexpr uint32_t TMEM_COLS = MX ? 512 : 2 * BN;       // two accumulator buffers (MX: accumulators + scales)
     // pair variant: rank of this CTA in its cluster of two; rank 0 leads (issues the MMAs, owns the
     // full and accumulator-empty barriers that both CTAs signal)
     const uint32_t rank = TWO ? cluster_ctarank() : 0u;
@@ -318,6 +355,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if constexpr (TWO) cluster_sync_all();       // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if constexpr (MX) {
+        // unit scales: every byte of 32 columns in all 128 lanes is UE8M0 127 = 2^0 (A's scales are read
+        // from the first 16 columns, B's from the second 16)
+        if (warp >= 2 && warp < 6) {
+            const uint32_t t_sf = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + SF_COL;
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) tmem_st4(t_sf + (uint32_t)c, 0x7F7F7F7Fu);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        tc_fence_before();
+        __syncthreads();
+        if constexpr (TWO) cluster_sync_all();   // the leader's MMAs read the scales of both CTAs
+        tc_fence_after();
+    }
     pdl_wait();     // set-up above overlaps the previous kernel; operands and outputs are touched only from here
 
     const int num_m = (p.M + TILE_M - 1) / TILE_M;
@@ -363,14 +414,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0 && leader) {
-            constexpr uint32_t idesc = F16 ? make_idesc_bf16(TILE_M, BN) : make_idesc_i8(TILE_M, BN);
+            constexpr uint32_t idesc = MX ? make_idesc_mxf4(TILE_M, BN) : F16 ? make_idesc_bf16(TILE_M, BN) : make_idesc_i8(TILE_M, BN);
             int stage = 0;
             uint32_t phase = 0;
             int t = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
-                const int buf = t & 1;
-                const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
+                const int buf = NBUF == 2 ? (t & 1) : 0;
+                const uint32_t bphase = (uint32_t)(NBUF == 2 ? (t >> 1) : t) & 1u;
                 ok = mbar_wait(smem_u32(&tempty_bar[buf]), bphase ^ 1u, abort_flag, p.status, ST_MMA);
                 if (!ok) break;
                 tc_fence_after();
@@ -388,7 +439,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const uint64_t ad = a_desc + (uint64_t)(kk * (UMMA_K >> 4));
                         const uint64_t bd = b_desc + (uint64_t)(kk * (UMMA_K >> 4));
                         const uint32_t accum = (kb | kk) != 0 ? 1u : 0u;
-                        if constexpr (F16) {      // 32 bytes of K = 16 bfloat16 per instruction
+                        if constexpr (MX) {       // 32 bytes of K = 64 E2M1 per instruction
+                            if constexpr (TWO) umma_mxf4_pair(d_tmem, ad, bd, idesc, accum, tmem_base + SF_COL, tmem_base + SF_COL + 16);
+                            else umma_mxf4(d_tmem, ad, bd, idesc, accum, tmem_base + SF_COL, tmem_base + SF_COL + 16);
+                        } else if constexpr (F16) {      // 32 bytes of K = 16 bfloat16 per instruction
                             if constexpr (TWO) umma_bf16_pair(d_tmem, ad, bd, idesc, accum);
                             else umma_bf16(d_tmem, ad, bd, idesc, accum);
                         } else {
@@ -426,13 +480,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
             const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
             const int n0 = (tile / num_m) * BN;
-            const int buf = t & 1;
-            const uint32_t bphase = (uint32_t)(t >> 1) & 1u;
+            const int buf = NBUF == 2 ? (t & 1) : 0;
+            const uint32_t bphase = (uint32_t)(NBUF == 2 ? (t >> 1) : t) & 1u;
             // stage this tile's column scales (and column corrections) in shared memory; the
             // buffer of tile t was last read during tile t-2, which every warp left before it
             // arrived at the barrier of tile t-1
-            float *swt = sw_tile + buf * BN;
-            int32_t *cbt = cb_tile + buf * BN;
+            float *swt = sw_tile + (t & 1) * BN;
+            int32_t *cbt = cb_tile + (t & 1) * BN;
             for (int c = ep_tid; c < BN; c += 32 * EPI_WARPS) {
                 const int col = n0 + c;
                 if (!BWD) swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
@@ -445,7 +499,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool fold = !CORR && !p.acc;
             float sxr = WO ? 1.0f : (!BWD && row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
             if (fold) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.sh) << 23));
-            if (p.ysh) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.ysh) << 23));
             int rsa = 0;
             if (CORR) rsa = (row_ok && p.rs_a) ? p.ca * __ldg(p.rs_a + row) + p.ck : p.ck;
             ok = mbar_wait(smem_u32(&tfull_bar[buf]), bphase, abort_flag, p.status, ST_EPILOGUE);
@@ -533,11 +586,26 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int j = 0; j < 32; ++j)
                             rc[j] = (uint32_t)((int32_t)((uint32_t)p.mul * rc[j] + (uint32_t)rsa +
                                                          (uint32_t)cbt[cbase + c0 + j]) >> p.sh);
-                    } else if (!fold) {
+                    } else if (!MX && !fold) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) rc[j] = (uint32_t)((int32_t)rc[j] >> p.sh);
                     }
-                    if (!BWD && p.acc && row_ok) {
+                    if (MX && p.acc && row_ok) {
+                        // acc4 = 4 * sum v_x v_w: the accumulator is an exact multiple of 1/4
+                        int32_t *dst = p.acc + (long long)row * p.N + col0;
+                        if (vec_acc && full) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<int4 *>(dst + j) =
+                                    make_int4(__float2int_rn(__uint_as_float(rc[j]) * 4.0f), __float2int_rn(__uint_as_float(rc[j + 1]) * 4.0f),
+                                              __float2int_rn(__uint_as_float(rc[j + 2]) * 4.0f), __float2int_rn(__uint_as_float(rc[j + 3]) * 4.0f));
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = __float2int_rn(__uint_as_float(rc[j]) * 4.0f);
+                        }
+                    }
+                    if (!MX && !BWD && p.acc && row_ok) {
                         int32_t *dst = p.acc + (long long)row * p.N + col0;
                         if (vec_acc && full) {
 #pragma unroll
@@ -555,7 +623,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const float2 *sw2 = reinterpret_cast<const float2 *>(swt + cbase + c0);
 #pragma unroll
                         for (int j = 0; j < (BWD ? 0 : 32); j += 2) {
-                            const float2 a2 = WO ? make_float2(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]))
+                            const float2 a2 = (WO || MX) ? make_float2(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]))
                                                  : make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
                             const float2 y2 = __fmul2_rn(__fmul2_rn(sx2, sw2[j >> 1]), a2);
                             rc[j] = __float_as_uint(y2.x);
@@ -697,22 +765,6 @@ __global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits,
     }
 }
 
-// E2M1 codes -> int8 operand values 2 v, 32 elements per thread.
-__global__ void unpack_fp4_kernel(const uint8_t *__restrict__ codes, long long n_groups, int8_t *__restrict__ out) {
-    pdl_launch_dependents();
-    pdl_wait();
-    for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n_groups;
-         g += (long long)gridDim.x * blockDim.x) {
-        const uint4 c = __ldg(reinterpret_cast<const uint4 *>(codes) + g);
-        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
-        uint32_t o[8];
-        fp4_operand_from_code_words(w, o);
-        uint4 *dst = reinterpret_cast<uint4 *>(out + g * 32);
-        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-    }
-}
-
 // Row sums of an int8 matrix [rows x K]: one warp per row.
 __global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, int K, int32_t *__restrict__ out) {
     pdl_launch_dependents();
@@ -823,17 +875,13 @@ Workspace carve_workspace(void *base, int64_t M, int64_t N, int64_t K) {
 }
 
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out, int32_t *rowsum,
-                  cudaStream_t st, int grid) {
+                  cudaStream_t st) {
     if (rows == 0) return QUEST_OK;
     const long long n_groups = rows * K / 32;
     const int threads = 256;
     long long blocks = (n_groups + threads - 1) / threads;
     if (blocks > 148 * 16) blocks = 148 * 16;
     cudaError_t e;
-    if (grid == GRID_FP4) {
-        e = launch_pdl(unpack_fp4_kernel, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, n_groups, out);
-        return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
-    }
     switch (container_bits(bits)) {
         case 1: e = launch_pdl(unpack_codes_kernel<1>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
         case 2: e = launch_pdl(unpack_codes_kernel<2>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
@@ -855,7 +903,7 @@ int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cu
 int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
                 int bits_x, int bits_w, const float *sx, const float *sw,
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
-                int32_t *acc, cudaStream_t st, int grid) {
+                int32_t *acc, cudaStream_t st) {
     if (M == 0 || N == 0) return QUEST_OK;
     // operand value v relates to the grid value c by v = 2^(7-b) c below 8 bits and c = 2v + 1 at 8 bits
     const bool x8 = bits_x == 8, w8 = bits_w == 8;
@@ -866,10 +914,6 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
     else if (x8 && w8) { p.mul = 4; p.ca = 2; p.cb = 2; p.ck = (int)K; p.sh = 0; }
     else if (x8) { p.mul = 2; p.ca = 0; p.cb = 1; p.ck = 0; p.sh = 7 - bits_w; }   // 2 sum v_x op_w + sum op_w
     else { p.mul = 2; p.ca = 1; p.cb = 0; p.ck = 0; p.sh = 7 - bits_x; }
-    p.ysh = 0;
-    if (grid == GRID_FP4) {    // operands are 2 v: acc = 4 sum v_x v_w is reported as is, y takes the factor 1/4
-        p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; p.ysh = 2;
-    }
     p.rs_a = p.ca ? rs_a : nullptr;                      // row sums of the x operand bytes
     p.rs_b = p.cb ? rs_b : nullptr;                      // row sums of the w operand bytes
     p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr;
@@ -913,7 +957,7 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     GemmParams p;
     p.M = (int)I; p.N = (int)J; p.K = (int)(2 * Kc);
     p.sx = nullptr; p.sw = nullptr; p.rs_a = nullptr; p.rs_b = nullptr;
-    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; p.ysh = 0;
+    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
     p.y = out; p.y_dtype = out_dtype; p.ldy = J; p.acc = nullptr; p.mask = mask;
     const int64_t esz = out_dtype == QUEST_F32 ? 4 : 2;
     p.status = device_status_word();
@@ -937,13 +981,46 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     return launch_gemm_bn<128, 2, false, true>(tmA, tmB, tmY, p, st);
 }
 
+// FP4 grid on the native path: xq [M x K/2], wq [N x K/2] packed E2M1 codes as the quantizer writes them.
+int launch_gemm_mxfp4(const uint8_t *xq, const uint8_t *wq, const float *sx, const float *sw, int64_t M, int64_t N,
+                      int64_t K, void *y, int y_dtype, int64_t ldy, int32_t *acc4, cudaStream_t st) {
+    if (M == 0 || N == 0) return QUEST_OK;
+    GemmParams p;
+    p.M = (int)M; p.N = (int)N; p.K = (int)(K / 2);
+    p.sx = sx; p.sw = sw; p.rs_a = nullptr; p.rs_b = nullptr;
+    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc4; p.mask = nullptr;
+    p.status = device_status_word();
+    if (!p.status) return QUEST_ERR_CUDA;
+    const bool wide = N > 128;
+    const bool pair = wide && M > 128;
+    CUtensorMap tmA, tmB;
+    int s = make_operand_map(&tmA, reinterpret_cast<const int8_t *>(xq), M, K / 2, BM);
+    if (s) return s;
+    s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(wq), N, K / 2, pair ? 128 : wide ? 256 : 128);
+    if (s) return s;
+    const size_t esz = y_dtype == QUEST_F32 ? 4 : 2;
+    const bool yt = y && (reinterpret_cast<uintptr_t>(y) % 16 == 0) && ((size_t)ldy * esz % 16 == 0);
+    CUtensorMap tmY = tmA;
+    if (yt) {
+        s = make_output_map(&tmY, y, M, (int64_t)N * (int64_t)esz, (int64_t)ldy * (int64_t)esz);
+        if (s) return s;
+    }
+#define QUEST_GEMM_MX(BNV, TWOV) \
+    (yt ? launch_gemm_bn<BNV, 5, TWOV, true>(tmA, tmB, tmY, p, st) : launch_gemm_bn<BNV, 5, TWOV, false>(tmA, tmB, tmY, p, st))
+    if (pair) return QUEST_GEMM_MX(256, true);
+    if (wide) return QUEST_GEMM_MX(256, false);
+    return QUEST_GEMM_MX(128, false);
+#undef QUEST_GEMM_MX
+}
+
 int launch_gemm_bf16_scaled(const void *a, const void *b, const float *sw, int64_t M, int64_t N, int64_t K,
                             void *y, int y_dtype, int64_t ldy, cudaStream_t st) {
     if (M == 0 || N == 0) return QUEST_OK;
     GemmParams p;
     p.M = (int)M; p.N = (int)N; p.K = (int)(2 * K);
     p.sx = nullptr; p.sw = sw; p.rs_a = nullptr; p.rs_b = nullptr;
-    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; p.ysh = 0;
+    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
     p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = nullptr; p.mask = nullptr;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;

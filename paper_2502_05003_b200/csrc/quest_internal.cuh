@@ -116,12 +116,12 @@ struct QuantJob {
 int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
                     float trust_factor, cudaStream_t st, int grid = GRID_UNIFORM);
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out,
-                  int32_t *rowsum, cudaStream_t st, int grid = GRID_UNIFORM);
+                  int32_t *rowsum, cudaStream_t st);
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st);
 int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
                 int bits_x, int bits_w, const float *sx, const float *sw,
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
-                int32_t *acc, cudaStream_t st, int grid = GRID_UNIFORM);
+                int32_t *acc, cudaStream_t st);
 
 // Per-stage event timing (quest_stage_timing): bracket a stage of another translation unit.
 void *stage_begin(int id, cudaStream_t st);
@@ -130,6 +130,10 @@ void stage_end(void *scope);
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
                             const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st);
 
+// FP4 contraction on packed E2M1 codes (tcgen05 kind::mxf4, unit block scales): acc4 = 4 sum v_x v_w (int32),
+// y = sx sw sum v_x v_w.  xq, wq 16-byte aligned, K % 32 == 0.
+int launch_gemm_mxfp4(const uint8_t *xq, const uint8_t *wq, const float *sx, const float *sw, int64_t M, int64_t N,
+                      int64_t K, void *y, int y_dtype, int64_t ldy, int32_t *acc4, cudaStream_t st);
 // Orthonormal block Hadamard transform of every row (binary32 or bfloat16 in, binary32 or bfloat16 out).
 int launch_hadamard_rows(const void *in, int in_dtype, int64_t ld_in, int64_t rows, int64_t cols, int had_block,
                          void *out, int out_dtype, int64_t ld, cudaStream_t st);

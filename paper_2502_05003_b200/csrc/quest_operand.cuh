@@ -87,31 +87,10 @@ __device__ __forceinline__ void operand_from_code_words(const uint32_t (&w)[CB],
 }
 
 // FP4 (E2M1) codes: sign << 3 | magnitude index m, values +-{0, .5, 1, 1.5, 2, 3, 4, 6}.
-// Twice the magnitude is an integer: m for m < 2, else (2 + (m & 1)) << ((m >> 1) - 1).
-__device__ __forceinline__ int e2m1_twice_magnitude(int m) {
-    const int e = m >> 1;
-    return e ? (2 + (m & 1)) << (e - 1) : m;
-}
 __device__ __forceinline__ float e2m1_value(int code) {
     const int m = code & 7, e = m >> 1;
     const float mag = e ? __uint_as_float(((uint32_t)(126 + e) << 23) | ((uint32_t)(m & 1) << 22)) : 0.5f * (float)m;
     return (code & 8) ? -mag : mag;
-}
-// Four E2M1 codes (16 bits, element 0 in the low nibble) -> four operand bytes 2 v (|2v| <= 12): one
-// byte permute looks the doubled magnitudes up in an 8-entry table, a second one picks each byte from
-// the magnitudes or from their negation according to the code's sign bit.
-__device__ __forceinline__ uint32_t fp4_operand4(uint32_t c16) {
-    const uint32_t mag = __byte_perm(0x03020100u, 0x0C080604u, c16 & 0x7777u);
-    const uint32_t neg = (0x80808080u - mag) ^ 0x80808080u;            // per byte -mag, no carries between bytes
-    return __byte_perm(mag, neg, 0x3210u + ((c16 & 0x8888u) >> 1));
-}
-// 32 consecutive E2M1 codes (4 words) -> 32 operand bytes in element order.
-__device__ __forceinline__ void fp4_operand_from_code_words(const uint32_t (&w)[4], uint32_t (&o)[8]) {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        o[2 * q] = fp4_operand4(w[q] & 0xFFFFu);
-        o[2 * q + 1] = fp4_operand4(w[q] >> 16);
-    }
 }
 
 // Sum of the four signed bytes of a word.

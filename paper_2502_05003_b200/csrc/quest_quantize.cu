@@ -446,10 +446,10 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                     }
                 }
             }
+            if constexpr (GRID == GRID_UNIFORM) {              // the FP4 codes are themselves the tensor-core operand
             if (FAST || tn.op8) {
                 uint32_t o[8];
-                if constexpr (GRID == GRID_FP4) fp4_operand_from_code_words(w, o);
-                else operand_from_code_words<CB>(w, a.bits, o);
+                operand_from_code_words<CB>(w, a.bits, o);
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -457,6 +457,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
 #pragma unroll
                     for (int q = 0; q < 8; ++q) rsum += sum_bytes_s8(o[q]);
                 }
+            }
             }
         }
     }

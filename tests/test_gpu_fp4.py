@@ -85,6 +85,27 @@ def test_gemm_accumulators_bit_exact(M, N, K):
     assert quest.quest_device_status() == 0
 
 
+def test_gemm_accumulators_exact_at_the_largest_sum():
+    # every product is +36 (6 x 6) or -36 over the longest supported row: |acc4| = 4 * 36 * K = 9.4 M < 2^24,
+    # the largest value the binary32 accumulators of the FP4 tensor-core path must hold exactly
+    import paper_2502_05003_b200 as quest
+    M, N, K = 130, 136, 65504
+    xq = np.full((M, K // 2), 0x77, np.uint8)               # +6, +6
+    xq[1::2] = 0xF7                                          # rows alternate: (+6, -6) pairs cancel
+    xq[2::3, : K // 4] = 0xFF                                # and some rows start with -6
+    wq = np.full((N, K // 2), 0x77, np.uint8)
+    wq[::5] = 0xFF
+    ones_m, ones_n = np.ones(M, np.float32), np.ones(N, np.float32)
+    d = lambda a: torch.from_numpy(a).cuda()
+    y, acc = quest.quest_lowbit_gemm_fp4(d(xq), d(ones_m), d(wq), d(ones_n), K, out_dtype=torch.float32, want_acc=True)
+    torch.cuda.synchronize()
+    ref = qo.gemm_acc_fp4(xq, wq, K)
+    assert np.abs(ref).max() == 4 * 36 * K
+    assert np.array_equal(acc.cpu().numpy(), ref)
+    assert np.array_equal(y.cpu().numpy().astype(np.float64) * 4.0, ref.astype(np.float64))
+    assert quest.quest_device_status() == 0
+
+
 @pytest.mark.parametrize("g", [128, 2048])
 def test_linear_fwd_config2(g):
     import paper_2502_05003_b200 as quest
