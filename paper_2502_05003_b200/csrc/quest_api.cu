@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "quest_internal.cuh"
+#include "quest_operand.cuh"
 
 namespace quest {
 
@@ -266,8 +267,9 @@ int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
     const bool need_rs_b = bits_x == 8;
     {
         StageScope scope(QUEST_STAGE_UNPACK, st);
-        if ((s = launch_unpack(xq, bits_x, M, K, ws.a8, need_rs_a ? ws.rs_a : nullptr, st))) return s;
-        if ((s = launch_unpack(wq, bits_w, N, K, ws.b8, need_rs_b ? ws.rs_b : nullptr, st))) return s;
+        const bool e4 = e2m1_operands(bits_x, bits_w);
+        if ((s = launch_unpack(xq, bits_x, M, K, ws.a8, need_rs_a ? ws.rs_a : nullptr, st, e4))) return s;
+        if ((s = launch_unpack(wq, bits_w, N, K, ws.b8, need_rs_b ? ws.rs_b : nullptr, st, e4))) return s;
     }
     StageScope scope(QUEST_STAGE_GEMM, st);
     return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits_x, bits_w, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc,
@@ -303,7 +305,7 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
             if ((s = launch_quantize(&jx, 1, dtype, K, bits, had_block, trust_factor, st))) return s;
         }
         StageScope scope(QUEST_STAGE_UNPACK, st);
-        if ((s = launch_unpack(wq, bits, N, K, ws.b8, need_rs ? ws.rs_b : nullptr, st))) return s;
+        if ((s = launch_unpack(wq, bits, N, K, ws.b8, need_rs ? ws.rs_b : nullptr, st, e2m1_operands(bits, bits)))) return s;
     } else {
         StageScope scope(QUEST_STAGE_QUANT_X, st);
         const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, ws.b8, need_rs ? ws.rs_b : nullptr}};
@@ -351,7 +353,7 @@ int quest_lowbit_gemm_fp4(const uint8_t *xq, const float *sx, const uint8_t *wq,
     (void)workspace;
     (void)workspace_bytes;
     StageScope scope(QUEST_STAGE_GEMM, st);
-    return launch_gemm_mxfp4(xq, wq, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc4, st);
+    return launch_gemm_e2m1(xq, wq, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc4, 4, st);
 }
 
 int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
@@ -384,7 +386,7 @@ int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int
         }
     }
     StageScope scope(QUEST_STAGE_GEMM, st);
-    return launch_gemm_mxfp4(xq, wq, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);
+    return launch_gemm_e2m1(xq, wq, sx, sw, M, N, K, y, y_dtype, N, nullptr, 4, st);
 }
 
 }  // extern "C"

@@ -11,7 +11,9 @@
 // c_x . c_w = 4 v_x.v_w + 2 sum(v_x) + 2 sum(v_w) + K exactly from per-row sums.
 //
 // The FP4 grid (Section 4.4) has a native operand type: its packed E2M1 codes feed tcgen05.mma
-// kind::mxf4 directly (MODE 5 below), with all block scales 2^0.
+// kind::mxf4 directly (MODE 5 below), with all block scales 2^0.  So do the one- and two-bit uniform
+// grids, whose values +-1 and +-3 are E2M1 numbers: when both operands have at most two bits the
+// workspace holds E2M1 nibbles and the same mode runs the contraction at twice the int8 rate.
 //
 // Two launch shapes of one kernel template.  TWO = false: one CTA per SM, persistent over 128 x BN
 // output tiles.  TWO = true: clusters of two CTAs (tcgen05 cta_group::2) persistent over 256 x 256
@@ -591,18 +593,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int j = 0; j < 32; ++j) rc[j] = (uint32_t)((int32_t)rc[j] >> p.sh);
                     }
                     if (MX && p.acc && row_ok) {
-                        // acc4 = 4 * sum v_x v_w: the accumulator is an exact multiple of 1/4
+                        // the accumulator is exact: an integer (uniform grids) or a multiple of 1/4 (FP4 grid, mul = 4)
                         int32_t *dst = p.acc + (long long)row * p.N + col0;
+                        const float am = (float)p.mul;
                         if (vec_acc && full) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
                                 *reinterpret_cast<int4 *>(dst + j) =
-                                    make_int4(__float2int_rn(__uint_as_float(rc[j]) * 4.0f), __float2int_rn(__uint_as_float(rc[j + 1]) * 4.0f),
-                                              __float2int_rn(__uint_as_float(rc[j + 2]) * 4.0f), __float2int_rn(__uint_as_float(rc[j + 3]) * 4.0f));
+                                    make_int4(__float2int_rn(__uint_as_float(rc[j]) * am), __float2int_rn(__uint_as_float(rc[j + 1]) * am),
+                                              __float2int_rn(__uint_as_float(rc[j + 2]) * am), __float2int_rn(__uint_as_float(rc[j + 3]) * am));
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) dst[j] = __float2int_rn(__uint_as_float(rc[j]) * 4.0f);
+                                if (col0 + j < p.N) dst[j] = __float2int_rn(__uint_as_float(rc[j]) * am);
                         }
                     }
                     if (!MX && !BWD && p.acc && row_ok) {
@@ -765,6 +768,22 @@ __global__ void unpack_codes_kernel(const uint8_t *__restrict__ codes, int bits,
     }
 }
 
+// Packed one- or two-bit codes -> E2M1 nibble operands (quest_operand.cuh), 32 elements per thread.
+template <int CB>
+__global__ void unpack_codes_e2m1_kernel(const uint8_t *__restrict__ codes, long long n_groups, uint8_t *__restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    for (long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x; g < n_groups;
+         g += (long long)gridDim.x * blockDim.x) {
+        uint32_t w[CB];
+#pragma unroll
+        for (int q = 0; q < CB; ++q) w[q] = __ldg(reinterpret_cast<const uint32_t *>(codes) + g * CB + q);
+        uint32_t o[4];
+        e2m1_operand_from_code_words<CB>(w, o);
+        *reinterpret_cast<uint4 *>(out + g * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 // Row sums of an int8 matrix [rows x K]: one warp per row.
 __global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, int K, int32_t *__restrict__ out) {
     pdl_launch_dependents();
@@ -875,13 +894,19 @@ Workspace carve_workspace(void *base, int64_t M, int64_t N, int64_t K) {
 }
 
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out, int32_t *rowsum,
-                  cudaStream_t st) {
+                  cudaStream_t st, bool e2m1) {
     if (rows == 0) return QUEST_OK;
     const long long n_groups = rows * K / 32;
     const int threads = 256;
     long long blocks = (n_groups + threads - 1) / threads;
     if (blocks > 148 * 16) blocks = 148 * 16;
     cudaError_t e;
+    if (e2m1) {                                       // bits <= 2: nibble operands, [rows x K/2] bytes
+        uint8_t *o4 = reinterpret_cast<uint8_t *>(out);
+        if (bits == 1) e = launch_pdl(unpack_codes_e2m1_kernel<1>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, n_groups, o4);
+        else e = launch_pdl(unpack_codes_e2m1_kernel<2>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, n_groups, o4);
+        return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+    }
     switch (container_bits(bits)) {
         case 1: e = launch_pdl(unpack_codes_kernel<1>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
         case 2: e = launch_pdl(unpack_codes_kernel<2>, dim3((unsigned)blocks), dim3(threads), 0, st, 1, codes, bits, n_groups, out); break;
@@ -905,6 +930,9 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
                 int64_t M, int64_t N, int64_t K, void *y, int y_dtype, int64_t ldy,
                 int32_t *acc, cudaStream_t st) {
     if (M == 0 || N == 0) return QUEST_OK;
+    if (e2m1_operands(bits_x, bits_w))               // both operands are E2M1 nibbles of the grid values
+        return launch_gemm_e2m1(reinterpret_cast<const uint8_t *>(a8), reinterpret_cast<const uint8_t *>(b8), sx, sw, M, N, K,
+                                y, y_dtype, ldy, acc, 1, st);
     // operand value v relates to the grid value c by v = 2^(7-b) c below 8 bits and c = 2v + 1 at 8 bits
     const bool x8 = bits_x == 8, w8 = bits_w == 8;
     GemmParams p;
@@ -981,15 +1009,16 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     return launch_gemm_bn<128, 2, false, true>(tmA, tmB, tmY, p, st);
 }
 
-// FP4 grid on the native path: xq [M x K/2], wq [N x K/2] packed E2M1 codes as the quantizer writes them.
-int launch_gemm_mxfp4(const uint8_t *xq, const uint8_t *wq, const float *sx, const float *sw, int64_t M, int64_t N,
-                      int64_t K, void *y, int y_dtype, int64_t ldy, int32_t *acc4, cudaStream_t st) {
+// Contraction of E2M1 nibble operands xq [M x K/2], wq [N x K/2] on the FP4 tensor-core path:
+// y = sx sw sum_k v_x v_w, acc = acc_mul * sum_k v_x v_w as int32 (the sum is exact in binary32).
+int launch_gemm_e2m1(const uint8_t *xq, const uint8_t *wq, const float *sx, const float *sw, int64_t M, int64_t N,
+                     int64_t K, void *y, int y_dtype, int64_t ldy, int32_t *acc, int acc_mul, cudaStream_t st) {
     if (M == 0 || N == 0) return QUEST_OK;
     GemmParams p;
     p.M = (int)M; p.N = (int)N; p.K = (int)(K / 2);
     p.sx = sx; p.sw = sw; p.rs_a = nullptr; p.rs_b = nullptr;
-    p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
-    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc4; p.mask = nullptr;
+    p.mul = acc_mul; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
     const bool wide = N > 128;

@@ -116,7 +116,7 @@ struct QuantJob {
 int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, int bits, int had_block,
                     float trust_factor, cudaStream_t st, int grid = GRID_UNIFORM);
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out,
-                  int32_t *rowsum, cudaStream_t st);
+                  int32_t *rowsum, cudaStream_t st, bool e2m1 = false);
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st);
 int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
                 int bits_x, int bits_w, const float *sx, const float *sw,
@@ -130,10 +130,11 @@ void stage_end(void *scope);
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
                             const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st);
 
-// FP4 contraction on packed E2M1 codes (tcgen05 kind::mxf4, unit block scales): acc4 = 4 sum v_x v_w (int32),
-// y = sx sw sum v_x v_w.  xq, wq 16-byte aligned, K % 32 == 0.
-int launch_gemm_mxfp4(const uint8_t *xq, const uint8_t *wq, const float *sx, const float *sw, int64_t M, int64_t N,
-                      int64_t K, void *y, int y_dtype, int64_t ldy, int32_t *acc4, cudaStream_t st);
+// Contraction of E2M1 nibble operands (tcgen05 kind::mxf4, unit block scales): acc = acc_mul * sum v_x v_w
+// (int32, exact), y = sx sw sum v_x v_w.  xq, wq 16-byte aligned, K % 32 == 0.  Serves the FP4 grid
+// (acc_mul = 4) and, inside launch_gemm, the one- and two-bit uniform grids (acc_mul = 1).
+int launch_gemm_e2m1(const uint8_t *xq, const uint8_t *wq, const float *sx, const float *sw, int64_t M, int64_t N,
+                     int64_t K, void *y, int y_dtype, int64_t ldy, int32_t *acc, int acc_mul, cudaStream_t st);
 // Orthonormal block Hadamard transform of every row (binary32 or bfloat16 in, binary32 or bfloat16 out).
 int launch_hadamard_rows(const void *in, int in_dtype, int64_t ld_in, int64_t rows, int64_t cols, int had_block,
                          void *out, int out_dtype, int64_t ld, cudaStream_t st);

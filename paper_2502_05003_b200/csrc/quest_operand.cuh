@@ -7,7 +7,8 @@
 // costs one shift and one three-input logic operation per four elements.  The contraction of two
 // such operands is 2^(14-bx-bw) * sum_k cx cw; the GEMM epilogue shifts it back (exact).
 // For b = 8 (|c| up to 255) the operand is v = k - 128 = k ^ 0x80 and the epilogue restores the
-// grid-value product from per-row sums of v.
+// grid-value product from per-row sums of v.  (When both operands have at most two bits the operand is
+// an E2M1 nibble instead: see e2m1_operands below.)
 #pragma once
 #include <stdint.h>
 
@@ -91,6 +92,38 @@ __device__ __forceinline__ float e2m1_value(int code) {
     const int m = code & 7, e = m >> 1;
     const float mag = e ? __uint_as_float(((uint32_t)(126 + e) << 23) | ((uint32_t)(m & 1) << 22)) : 0.5f * (float)m;
     return (code & 8) ? -mag : mag;
+}
+
+// The uniform grids of one and two bits are subsets of the E2M1 values (+-1; +-1, +-3), so when both
+// operands of a contraction have at most two bits their operand is the E2M1 nibble of the grid value
+// (two elements per byte, element 0 in the low nibble) and the contraction runs on the FP4 tensor-core
+// path at twice the int8 rate:  b = 1: k = 0, 1 -> 0xA (-1), 0x2 (+1);  b = 2: k = 0..3 -> 0xD (-3),
+// 0xA (-1), 0x2 (+1), 0x5 (+3).
+__host__ __device__ inline bool e2m1_operands(int bits_x, int bits_w) { return bits_x <= 2 && bits_w <= 2; }
+
+// 32 consecutive codes (CB = 1 or 2 words) -> 32 E2M1 nibbles in element order (4 words).
+template <int CB>
+__device__ __forceinline__ void e2m1_operand_from_code_words(const uint32_t (&w)[CB], uint32_t (&o)[4]) {
+    static_assert(CB == 1 || CB == 2, "only the one- and two-bit grids are E2M1 subsets");
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if constexpr (CB == 1) {
+            const uint32_t b = (w[0] >> (8 * q)) & 0xFFu;          // eight levels, one bit each
+            uint32_t t = (b | (b << 12)) & 0x000F000Fu;            // spread: bit j -> bit 0 of nibble j
+            t = (t | (t << 6)) & 0x03030303u;
+            t = (t | (t << 3)) & 0x11111111u;
+            o[q] = 0xAAAAAAAAu ^ (t << 3);                         // k = 1 clears the sign bit
+        } else {
+            const uint32_t h = (w[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;   // eight levels, two bits each
+            uint32_t t = (h | (h << 8)) & 0x00FF00FFu;             // spread: level j -> low bits of nibble j
+            t = (t | (t << 4)) & 0x0F0F0F0Fu;
+            t = (t | (t << 2)) & 0x33333333u;
+            const uint32_t x = (t ^ (t >> 1)) & 0x11111111u;       // k1 ^ k0: set for the inner levels (+-1)
+            const uint32_t k1 = (t >> 1) & 0x11111111u;
+            // sign = !k1; +-3 = 0b101 (bits 0 and 2) when the level bits agree, +-1 = 0b010 otherwise
+            o[q] = ((k1 ^ 0x11111111u) << 3) | ((x ^ 0x11111111u) * 5u) | (x << 1);
+        }
+    }
 }
 
 // Sum of the four signed bytes of a word.

@@ -447,7 +447,15 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 }
             }
             if constexpr (GRID == GRID_UNIFORM) {              // the FP4 codes are themselves the tensor-core operand
-            if (FAST || tn.op8) {
+            if constexpr (CB <= 2) {
+                // one- and two-bit grids: E2M1 nibbles for the FP4 tensor-core path, 16 bytes per 32 elements
+                if (FAST || tn.op8) {
+                    uint32_t o[4];
+                    e2m1_operand_from_code_words<CB>(w, o);
+                    *reinterpret_cast<uint4 *>(tn.op8 + row * (long long)(cols >> 1) + (long long)tr * (E / 2) + g32 * 16) =
+                        make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            } else if (FAST || tn.op8) {
                 uint32_t o[8];
                 operand_from_code_words<CB>(w, a.bits, o);
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
