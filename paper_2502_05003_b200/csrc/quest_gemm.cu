@@ -261,14 +261,14 @@ __device__ __forceinline__ void pin(uint32_t &v) { asm volatile("" : "+r"(v)::"m
 
 template <int BN, bool TWO>
 struct SmemLayout {
-    static constexpr int NSTAGES = TWO ? 4 : (BN == 256 ? 3 : STAGES);   // four stages already saturate the MMA pipe
+    static constexpr int NSTAGES = TWO ? 5 : (BN == 256 ? 3 : STAGES);   // a lone pair saturates with four; with every pair loading, the fifth is worth 9 % on large shapes
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_ROWS = TWO ? BN / 2 : BN;         // rows of B this CTA stages
     static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int BAR_OFFSET = NSTAGES * STAGE_BYTES;
     static constexpr int STG_OFFSET = BAR_OFFSET;            // [8 warps][SLABS][32 rows x 128 B] output staging
-    static constexpr int SLABS = (TWO || BN == 128) ? 2 : 1;
+    static constexpr int SLABS = (BN == 128) ? 2 : 1;           // what the stages leave room for
     static constexpr int STG_BYTES = EPI_WARPS * SLABS * 4096;
     static constexpr int BAR_OFFSET2 = STG_OFFSET + STG_BYTES;
     static constexpr int SW_OFFSET = BAR_OFFSET2 + 256;      // [2][BN] column scales
