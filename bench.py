@@ -2,7 +2,7 @@
 """Benchmark of the QuEST quantized-linear forward hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--had-block G]
-                    [--no-graph] [--pass backward|weight_only]
+                    [--no-graph] [--pass backward|weight_only] [--bits B]
 
 One "step" is one pass of the whole path (Algorithm 1: quantize X, quantize W, low-bit GEMM with
 the dequantising epilogue) through the C ABI call ``quest_linear_fwd`` on the 1.6B-scale layer:
@@ -60,7 +60,8 @@ def load_peaks():
 
 
 def workload_config(had_block: int) -> dict:
-    return {"workload": "config 2: W4A4 linear fwd, X[4096x2048] bf16 x W[2048x2048] bf16, b=4",
+    name = "config 2" if BITS == 4 else "config 3"
+    return {"workload": f"{name}: W{BITS}A{BITS} linear fwd, X[4096x2048] bf16 x W[2048x2048] bf16, b={BITS}",
             "tokens": TOKENS, "K": HIDDEN, "N": OUT, "bits": BITS, "had_block": had_block,
             "trust_factor": 1.0, "weights": "quantized every step (Algorithm 1 as written)"}
 
@@ -389,7 +390,9 @@ def run_gpu(args, rank: int, world: int, local: int):
 
     peaks = load_peaks()
     src = "of measured" if peaks["_source"] == "measured" else "of fallback"
-    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
+    # one- and two-bit codes run on the FP4 tensor-core path (nominal rate twice that of int8)
+    fp4_path = BITS <= 2
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16 * (2.0 if fp4_path else 1.0)
     gemm_ms = stage_ms["gemm"]
     gemm_tops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12 if gemm_ms else None
     qx_bytes, qw_bytes = quantizer_bytes(M, K, BITS), quantizer_bytes(N, K, BITS)
@@ -420,7 +423,7 @@ def run_gpu(args, rank: int, world: int, local: int):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * max_elapsed / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "e2m1" if fp4_path else "s8",
         "data": "synthetic",
         "config": dict(workload_config(g), parallelism=f"replicas x{world}",
                        l2="ring of %d buffer sets (%.0f MB) larger than L2; no flush" % (n_sets, n_sets * set_bytes / 1e6)),
@@ -429,15 +432,19 @@ def run_gpu(args, rank: int, world: int, local: int):
         "gpu_launches": 2 * args.steps,     # per step: one quantizer launch (x and w together), one GEMM launch
         "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
         "clocks": clocks.summary(),
-        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel (tcgen05 kind::i8)", "achieved": gemm_tops,
+        "roofline": {"bound": "tensor",
+                     "kernel": "gemm_i8_kernel<mode 5> (tcgen05 kind::mxf4 on E2M1 operands)" if fp4_path
+                               else "gemm_i8_kernel (tcgen05 kind::i8)",
+                     "achieved": gemm_tops,
                      "peak": int8_peak, "unit": "TOP/s", "frac": (gemm_tops / int8_peak) if gemm_tops else None,
-                     "peak_basis": f"2 x bf16 burst {src} ({peaks['bf16_tflops']} TFLOP/s)",
-                     "traffic": GEMM_DRAM_TRAFFIC_BYTES, "ms": gemm_ms,
+                     "peak_basis": f"{4 if fp4_path else 2} x bf16 burst {src} ({peaks['bf16_tflops']} TFLOP/s)",
+                     "traffic": GEMM_DRAM_TRAFFIC_BYTES if BITS == 4 else None, "ms": gemm_ms,
                      "library_int8_gemm_tops_same_shape": lib_tops},
         "roofline_quantizer": {"bound": "hbm", "kernel": "quantizer, x and w rows in one launch", "achieved": q_gbs,
                                "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": (q_gbs / peaks["hbm_gbs"]) if q_gbs else None, "peak_basis": src,
-                               "traffic": QUANT_DRAM_TRAFFIC_BYTES, "ms": q_ms, "algorithmic_bytes": q_bytes,
+                               "traffic": QUANT_DRAM_TRAFFIC_BYTES if BITS == 4 else None, "ms": q_ms,
+                               "algorithmic_bytes": q_bytes,
                                # the kernel is bound by instruction issue, not HBM: the same launch against the
                                # issue rate 148 SMs x 4 schedulers x 32 lanes x SM clock
                                "alu": (lambda mhz: {"bound": "alu", "unit": "T thread-instr/s",
@@ -446,7 +453,7 @@ def run_gpu(args, rank: int, world: int, local: int):
                                                     "frac": QUANT_INSTR_PER_ELEMENT * (M + N) * K / (q_ms * 1e-3)
                                                             / (148 * 4 * 32 * mhz * 1e6),
                                                     "instr_per_element": QUANT_INSTR_PER_ELEMENT})(
-                                   clocks.summary()["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)) if q_ms else None},
+                                   clocks.summary()["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)) if (q_ms and BITS == 4) else None},
         "stage_ms": stage_ms,
         "cpu_baseline": {"value": sample / o_dt, "unit": UNIT, "cores": o_threads, "kind": "oracle",
                          "sample": f"{sample} of {TOKENS} token rows against the full W, one pass"},
@@ -708,10 +715,16 @@ def main():
     ap.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward", "weight_only"],
                     help="forward: Algorithm 1, the headline metric (default); backward: Algorithm 2 on the same layer; "
                          "weight_only: the W4A16 forward of Section 4.5 on the same layer")
+    ap.add_argument("--bits", type=int, default=4, choices=[1, 2, 3, 4, 8],
+                    help="width b of weights and activations for the forward pass (default 4, the headline; "
+                         "1 and 2 are the W1A1 / W2A2 variants of the same layer)")
     ap.add_argument("--ref-tokens", type=int, default=0,
                     help="token rows in the CPU oracle's bounded sample (0: the full 4096 for the "
                          "cpu_baseline leg; sized to about a minute in total for --impl reference)")
     args = ap.parse_args()
+    global BITS, METRIC
+    BITS = args.bits
+    METRIC = f"QuEST W{BITS}A{BITS} linear fwd tokens/s"
     rank, world, local = init_ranks(args.gpus)
     if args.impl == "reference":
         run_reference(args, rank)
