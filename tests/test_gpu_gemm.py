@@ -60,7 +60,29 @@ def test_w4a4_shapes(M, N, K, out_dtype):
     run_case(M, N, K, 4, 4, out_dtype, seed=M + N + K)
 
 
-@pytest.mark.parametrize("bx,bw", [(1, 1), (2, 2), (3, 3), (8, 8), (4, 8), (8, 4), (1, 4), (5, 7)])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (1, 8, 32), (37, 29, 96), (130, 260, 160), (300, 1000, 2048),
+                                   (513, 136, 5504), (64, 7, 64)])
+@pytest.mark.parametrize("bits", [1, 2])
+def test_one_and_two_bit_codes_on_the_fp4_path(M, N, K, bits):
+    # both operands at most two bits wide: E2M1 nibble operands, kind::mxf4 contraction, exact integer sums
+    run_case(M, N, K, bits, bits, torch.float32, seed=M + N + K + bits)
+
+
+def test_two_bit_codes_at_the_longest_row_and_config3_size():
+    import paper_2502_05003_b200 as quest
+    K = 65504
+    top = np.full((130, K // 4), 0xFF, np.uint8)        # every level 3 -> c = +3
+    bot = np.zeros((136, K // 4), np.uint8)             # every level 0 -> c = -3
+    ones = torch.ones(136, dtype=torch.float32, device="cuda")
+    _, acc = quest.quest_lowbit_gemm(torch.from_numpy(top).cuda(), ones[:130], 2, torch.from_numpy(bot).cuda(), ones, 2,
+                                     K, want_y=False, want_acc=True)
+    assert bool((acc == -9 * K).all())
+    rows = np.sort(np.random.default_rng(3).choice(4096, size=64, replace=False))
+    run_case(4096, 2048, 2048, 1, 1, torch.bfloat16, seed=4, sample_rows=rows)
+    run_case(4096, 2048, 2048, 2, 2, torch.bfloat16, seed=5, sample_rows=rows)
+
+
+@pytest.mark.parametrize("bx,bw", [(1, 1), (2, 2), (1, 2), (2, 1), (2, 3), (3, 3), (8, 8), (4, 8), (8, 4), (1, 4), (5, 7)])
 def test_bit_width_combinations(bx, bw):
     K = 1024 if max(bx, bw) < 8 else 512
     run_case(200, 328, K, bx, bw, torch.float32, seed=bx * 9 + bw)
