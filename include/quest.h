@@ -153,6 +153,13 @@ int quest_lowbit_gemm_static(const uint8_t *xq, const float *sx, int bits_x,
  *   wq, sw, mw             the same for w.  If w_is_cached != 0, w may be NULL and wq/sw are
  *                          INPUTS produced by an earlier call with the same bits and had_block
  *                          (the inference pipeline of Section 5); mw is then untouched
+ *   w_is_cached            0: quantize w.  1: take wq/sw and unpack wq into the workspace.
+ *                          2: as 1, and the workspace already holds the tensor-core operand of this
+ *                          w: it was filled by an earlier call (w_is_cached 0 or 1) with the same
+ *                          workspace pointer, w, N, K and bits, and nothing else wrote the workspace
+ *                          since.  M may differ between those calls (w's operand sits at the start of
+ *                          the workspace); the workspace must be large enough for this call's M.
+ *                          Other values: QUEST_ERR_SHAPE.
  *   workspace              as for quest_lowbit_gemm with bits_x = bits_w = bits
  */
 int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,

@@ -165,7 +165,9 @@ def quest_linear_fwd(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int
     """Algorithm 1: returns {"y", "xq", "sx", "mx", "wq", "sw", "mw"}.
 
     ``saved`` may carry preallocated output tensors under those keys; ``w_cached`` = {"wq", "sw"}
-    from an earlier call skips the weight quantization (then ``w`` may be None).
+    from an earlier call skips the weight quantization (then ``w`` may be None).  With
+    ``w_cached["operand_in_workspace"]`` true the call also skips unpacking ``wq``: ``workspace``
+    must be the tensor an earlier call for the same w used, untouched since (M may differ).
     """
     _require_cuda(x, w, y, workspace)
     M, K = x.shape
@@ -199,7 +201,8 @@ def quest_linear_fwd(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int
     st = _lib.load().quest_linear_fwd(
         _p(x), _p(w), _dtype_code(x), M, N, K, bits, had_block, ctypes.c_float(trust_factor),
         _p(y), _dtype_code(y), _p(out["xq"]), _p(out["sx"]), _p(out["mx"]),
-        _p(out["wq"]), _p(out["sw"]), _p(out["mw"]), 1 if w_cached is not None else 0,
+        _p(out["wq"]), _p(out["sw"]), _p(out["mw"]),
+        0 if w_cached is None else (2 if w_cached.get("operand_in_workspace") else 1),
         _p(workspace), workspace.numel(), _stream())
     _lib.check(st)
     out["y"] = y

@@ -284,6 +284,7 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
                      void *workspace, size_t workspace_bytes, void *stream) {
     if (!y || !xq || !sx || !wq || !sw) return QUEST_ERR_NULL;
     if (!w_is_cached && !w) return QUEST_ERR_NULL;
+    if (w_is_cached < 0 || w_is_cached > 2) return QUEST_ERR_SHAPE;
     if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
     int s = validate_gemm_shape(M, N, K, bits, bits);
     if (s) return s;
@@ -304,8 +305,10 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
             StageScope scope(QUEST_STAGE_QUANT_X, st);
             if ((s = launch_quantize(&jx, 1, dtype, K, bits, had_block, trust_factor, st))) return s;
         }
-        StageScope scope(QUEST_STAGE_UNPACK, st);
-        if ((s = launch_unpack(wq, bits, N, K, ws.b8, need_rs ? ws.rs_b : nullptr, st, e2m1_operands(bits, bits)))) return s;
+        if (w_is_cached != 2) {      // 2: the workspace still holds w's operand from an earlier call
+            StageScope scope(QUEST_STAGE_UNPACK, st);
+            if ((s = launch_unpack(wq, bits, N, K, ws.b8, need_rs ? ws.rs_b : nullptr, st, e2m1_operands(bits, bits)))) return s;
+        }
     } else {
         StageScope scope(QUEST_STAGE_QUANT_X, st);
         const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, ws.b8, need_rs ? ws.rs_b : nullptr}};

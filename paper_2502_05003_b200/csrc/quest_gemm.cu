@@ -877,18 +877,20 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
 
 }  // namespace
 
+// The operand of w and its row sums come first, so that their place does not depend on M: a caller
+// that keeps the workspace can reuse w's operand across calls with different numbers of rows of x.
 Workspace carve_workspace(void *base, int64_t M, int64_t N, int64_t K) {
     Workspace w;
     size_t off = 0;
     uint8_t *b = reinterpret_cast<uint8_t *>(base);
-    w.a8 = reinterpret_cast<int8_t *>(b + off);
-    off += align_up((size_t)(M * K), 256);
     w.b8 = reinterpret_cast<int8_t *>(b + off);
     off += align_up((size_t)(N * K), 256);
-    w.rs_a = reinterpret_cast<int32_t *>(b + off);
-    off += align_up((size_t)M * 4, 256);
     w.rs_b = reinterpret_cast<int32_t *>(b + off);
     off += align_up((size_t)N * 4, 256);
+    w.a8 = reinterpret_cast<int8_t *>(b + off);
+    off += align_up((size_t)(M * K), 256);
+    w.rs_a = reinterpret_cast<int32_t *>(b + off);
+    off += align_up((size_t)M * 4, 256);
     w.bytes = off;
     return w;
 }

@@ -140,3 +140,23 @@ def test_two_streams_share_no_hidden_state():
             for k in ("y", "xq", "mx", "wq", "mw", "sx", "sw"):
                 assert torch.equal(outs[i][k], serial[i][k]), (rep, i, k)
     assert quest.quest_device_status() == 0
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_cached_weight_operand_is_reused_across_calls_with_other_row_counts(bits):
+    """w_is_cached = 2: the operand of w left in the workspace by an earlier call serves later calls."""
+    import paper_2502_05003_b200 as quest
+    rng = np.random.default_rng(40 + bits)
+    N, K, g = 264, 512, 128
+    w = torch.from_numpy(synth.f32_to_bf16_bits((rng.standard_normal((N, K)) * 0.02).astype(np.float32))).view(torch.bfloat16).cuda()
+    xs = [torch.from_numpy(synth.f32_to_bf16_bits(rng.standard_normal((M, K)).astype(np.float32))).view(torch.bfloat16).cuda()
+          for M in (300, 130, 520)]
+    ws = quest.alloc_workspace(520, N, K, bits, bits)
+    first = quest.quest_linear_fwd(xs[0], w, bits, g, workspace=ws)
+    cached = {"wq": first["wq"], "sw": first["sw"], "operand_in_workspace": True}
+    for x in xs[1:]:
+        got = quest.quest_linear_fwd(x, None, bits, g, w_cached=cached, workspace=ws)
+        ref = quest.quest_linear_fwd(x, w, bits, g)
+        torch.cuda.synchronize()
+        assert torch.equal(got["y"], ref["y"]) and torch.equal(got["xq"], ref["xq"])
+    assert quest.quest_device_status() == 0
