@@ -709,7 +709,9 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
         const int T = (int)(cols / E);
         int S;
         if (T < 32) { S = 1; while (S < T) S <<= 1; } else { S = (T + 31) / 32 * 32; }
-        const int R = S >= 256 ? 1 : 256 / S;
+        // rows per CTA: 128-thread CTAs for the 32-per-thread streaming kernel (eight per SM) measured 4-10 % faster
+        // than 256-thread ones: finer work units at the tail and fewer warps behind each CTA-wide barrier
+        const int R = (stream32 && S <= 128) ? 128 / S : (S >= 256 ? 1 : 256 / S);
         const int threads = R * S;
         const int warps = (threads + 31) / 32;
         const size_t smem = had_block >= 64 * E ? sizeof(float) * E * (size_t)threads : sizeof(float) * (size_t)warps;
@@ -750,7 +752,7 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 int dev = 0, sms = 148;
                 cudaGetDevice(&dev);
                 cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-                const int per_sm = smem2 > 100 * 1024 ? 1 : (E == 64 ? 2 : 4);
+                const int per_sm = smem2 > 100 * 1024 ? 1 : (E == 64 ? 2 : (threads <= 128 ? 8 : 4));
                 const int total = nb[0] + nb[1];
                 const int g = total < sms * per_sm ? total : sms * per_sm;
                 bool fast = had_block == 128 && S >= 32 && bits < 8 && trust_factor >= 1.0f;
