@@ -354,7 +354,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                         t[2 * j + 1] = __fmul_rn(v[g32 * 16 + q * 4 + j].y, inv);
                     }
                     const uint32_t cw = cvt_e2m1x8(t);
-                    if (hh >= 1.0f) {
+                    if (FAST || hh >= 1.0f) {
                         // every element inside the grid is within one value unit of its point (exactly, the
                         // difference being exact); only saturated elements can fail: |t| - 6 > trust_factor
 #pragma unroll
@@ -663,13 +663,13 @@ static cudaError_t launch_rows_fp4(dim3 grid, int threads, size_t smem, cudaStre
     return launch_pdl(quantize_rows_kernel<BF16, 4, E, GRID_FP4>, grid, dim3(threads), smem, st, 1, a);
 }
 
-template <int E>
+template <int E, bool FAST>
 static cudaError_t launch_stream_fp4(int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                      int total_groups, int exchange_bytes) {
-    cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<4, E, false, GRID_FP4>,
+    cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<4, E, FAST, GRID_FP4>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
     if (e_ != cudaSuccess) return e_;
-    return launch_pdl(quantize_stream_kernel<4, E, false, GRID_FP4>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a,
+    return launch_pdl(quantize_stream_kernel<4, E, FAST, GRID_FP4>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a,
                       total_groups, exchange_bytes);
 }
 
@@ -760,10 +760,20 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                     const QuantTensor &t = a.t[j];
                     if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum && !t.rot && !t.cbf)) fast = false;
                 }
-                if (grid_kind == GRID_FP4)
-                    e = E == 64 ? launch_stream_fp4<64>(g, threads, smem2, st, a, total, exchange)
-                                : launch_stream_fp4<32>(g, threads, smem2, st, a, total, exchange);
-                else if (fast)
+                if (grid_kind == GRID_FP4) {
+                    // the FP4 codes are the GEMM operand themselves: the specialised path wants codes, scales, mask
+                    bool fast4 = had_block == 128 && S >= 32 && trust_factor >= 1.0f;
+                    for (int j = 0; j < 2; ++j) {
+                        const QuantTensor &t = a.t[j];
+                        if (t.rows > 0 && !(t.codes && t.scales && t.mask && !t.op8 && !t.rowsum && !t.rot && !t.cbf)) fast4 = false;
+                    }
+                    if (fast4)
+                        e = E == 64 ? launch_stream_fp4<64, true>(g, threads, smem2, st, a, total, exchange)
+                                    : launch_stream_fp4<32, true>(g, threads, smem2, st, a, total, exchange);
+                    else
+                        e = E == 64 ? launch_stream_fp4<64, false>(g, threads, smem2, st, a, total, exchange)
+                                    : launch_stream_fp4<32, false>(g, threads, smem2, st, a, total, exchange);
+                } else if (fast)
                     e = E == 64 ? launch_stream<64, true>(cb, g, threads, smem2, st, a, total, exchange)
                                 : launch_stream<32, true>(cb, g, threads, smem2, st, a, total, exchange);
                 else
