@@ -603,9 +603,9 @@ def run_backward(args, rank: int, world: int, local: int):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": dict(workload_config(g), workload="config 2, Algorithm 2 (backward): dy[4096x2048] bf16 -> dx, dw bf16",
                        l2="ring of %d buffer sets (%.0f MB) larger than L2" % (n_sets, n_sets * set_bytes / 1e6)),
-        "gpu_launches": 5 * steps, "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
+        "gpu_launches": 3 * steps, "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
         "clocks": clocks.summary(),
-        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel<mode 3> (tcgen05 kind::f16 bf16, fused mask + inverse Hadamard)",
+        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel<mode 3> (tcgen05 kind::f16 bf16, MN-major operands, fused mask + inverse Hadamard)",
                      "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": (tflops / peaks["bf16_tflops"]) if tflops else None,
                      "peak_basis": "bf16 burst " + ("of measured" if peaks["_source"] == "measured" else "of fallback"),

@@ -178,20 +178,19 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
  *
  * with the trust estimator of Section 3.2 applied in the Hadamard domain and IHT the inverse of
  * the orthonormal block Hadamard transform.  The two products run on the tensor cores with
- * bfloat16 operands and binary32 accumulation ("standard 16-bit precision", Section 3.3): the grid
- * values are exact in bfloat16 and the per-row scale of the quantized operand is folded into dL/dy
- * before it is rounded to bfloat16.
+ * bfloat16 operands and binary32 accumulation ("standard 16-bit precision", Section 3.3): dL/dy as
+ * given, the quantized operand dequantised to bfloat16 (scale * grid value, one rounding per element).
  *
  *   dy                 device, [M x N] bfloat16, dense, 16-byte aligned
  *   M, N, K            M, N > 0 and multiples of 8; 32 <= K <= 16384, K % 32 == 0
  *   bits, had_block    as in the forward call that produced the codes
  *   xq, sx, mx         device: codes [M x K], scales [M], trust mask [M x K/8] of x (forward outputs);
- *                      masks and sw 16-byte aligned, codes 4-byte aligned
+ *                      masks 16-byte aligned, codes 4-byte aligned
  *   wq, sw, mw         the same for w ([N x K])
  *   dx, dw             device out: [M x K] and [N x K], dense, out_dtype (QUEST_F32 or QUEST_BF16),
  *                      16-byte aligned; either may be NULL to skip that gradient
  *   workspace          device scratch of at least quest_bwd_workspace_bytes(M, N, K) bytes, 256-byte
- *                      aligned (bfloat16 operands and the masked binary32 products)
+ *                      aligned (dequantised bfloat16 operands and the masked binary32 products)
  */
 int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K, int bits, int had_block,
                      const uint8_t *xq, const float *sx, const uint8_t *mx,

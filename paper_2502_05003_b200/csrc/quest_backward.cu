@@ -3,16 +3,16 @@
 //   dL/dxq_h = dL/dy wq_h                      dL/dx = IHT(M(x_h; xq_h) * dL/dxq_h)
 //   dL/dwq_h = dL/dy^T xq_h                    dL/dw = IHT(M(w_h; wq_h) * dL/dwq_h)
 //
-// The products run in 16-bit precision on the tensor cores (Section 3.3, "Implementation"): the
-// integer grid values c = 2k - (2^b - 1) are exact in bfloat16, and the per-row scale of the
-// quantized operand is folded into dL/dy before it is rounded to bfloat16 (the scale multiplies
-// the contraction index, so it cannot be pulled out of the sum).  Stages:
-//   1. scale_dy_kernel        a1[m][n] = bf16(dy[m][n] sw[n])         (operand of line 2)
-//                             a2[n][m] = bf16(dy[m][n] sx[m])         (operand of line 4, transposed)
-//   2. codes_to_bf16_t_kernel ct[k][r] = bf16(c[r][k])  for w and x   (K-major operands)
-//   3. gemm (quest_gemm.cu, bfloat16 mode): masked binary32 products  d1 [M x K], d2 [N x K]
-//   4. iht_rows_kernel        block Hadamard transform, 1/sqrt(g), store in the output type
-//      (for blocks of 128 stages 3 and 4 are one kernel: the transform runs in the GEMM epilogue,
+// The products run in 16-bit precision on the tensor cores (Section 3.3, "Implementation").  dL/dy is
+// used as it is (bfloat16); the quantized operand is dequantised to bfloat16, xq_h = bf16(sx[m] c_x),
+// wq_h = bf16(sw[n] c_w) with c = 2k - (2^b - 1): one rounding per product.  Nothing is transposed: the
+// tensor cores read an operand whose memory rows run along the contraction index as an MN-major
+// operand (quest_gemm.cu).  Stages:
+//   1. dequant_codes_kernel   wq_h [N x K], xq_h [M x K] from the packed codes and scales
+//   2. gemm (bfloat16 mode)   d1[m][k] = M_x[m][k] sum_n dy[m][n] wq_h[n][k]   (dy K-major, wq_h MN-major)
+//                             d2[n][k] = M_w[n][k] sum_m dy[m][n] xq_h[m][k]   (dy and xq_h MN-major)
+//   3. iht_rows_kernel        block Hadamard transform, 1/sqrt(g), store in the output type
+//      (for blocks of 128 stages 2 and 3 are one kernel: the transform runs in the GEMM epilogue,
 //      where a thread holds exactly one block of its output row)
 #include <cuda_bf16.h>
 #include <math.h>
@@ -27,96 +27,45 @@ __device__ __forceinline__ uint16_t bf16_bits(float v) {
     return *reinterpret_cast<uint16_t *>(&h);
 }
 
-// dy [M x N] bfloat16 -> a1 [M x N] = dy * sw[n], a2 [N x M] = (dy * sx[m])^T, both rounded to bfloat16.
-// 64 x 64 tiles, 256 threads, 16-byte accesses on both sides (M and N are multiples of 8, so an
-// 8-element chunk is inside or outside the matrix as a whole).
-__global__ void __launch_bounds__(256)
-scale_dy_kernel(const uint16_t *__restrict__ dy, const float *__restrict__ sx, const float *__restrict__ sw,
-                int M, int N, uint16_t *__restrict__ a1, uint16_t *__restrict__ a2) {
-    __shared__ uint32_t tile[64][33];                          // [m][n pairs]; odd pitch keeps the transposed reads apart
-    pdl_launch_dependents();
-    pdl_wait();
-    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
-    const int t = threadIdx.x;
-    const int chunk = t & 7;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int ml = (t >> 3) + 32 * i;
-        const int m = m0 + ml, n = n0 + chunk * 8;
-        uint32_t q[4] = {0u, 0u, 0u, 0u};
-        if (m < M && n < N) {
-            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(dy + (long long)m * N + n));
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-            const float sxm = __ldg(sx + m);
-            const float4 s0 = __ldg(reinterpret_cast<const float4 *>(sw + n));
-            const float4 s1 = __ldg(reinterpret_cast<const float4 *>(sw + n + 4));
-            const float swn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-            uint32_t o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float lo = __uint_as_float(ww[j] << 16), hi = __uint_as_float(ww[j] & 0xFFFF0000u);
-                o[j] = (uint32_t)bf16_bits(lo * swn[2 * j]) | ((uint32_t)bf16_bits(hi * swn[2 * j + 1]) << 16);
-                q[j] = (uint32_t)bf16_bits(lo * sxm) | ((uint32_t)bf16_bits(hi * sxm) << 16);
-            }
-            *reinterpret_cast<uint4 *>(a1 + (long long)m * N + n) = make_uint4(o[0], o[1], o[2], o[3]);
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) tile[ml][chunk * 4 + j] = q[j];
-    }
-    __syncthreads();
-    const uint16_t *t16 = reinterpret_cast<const uint16_t *>(&tile[0][0]);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int nl = (t >> 3) + 32 * i;
-        const int n = n0 + nl, m = m0 + chunk * 8;
-        if (n < N && m < M) {
-            uint32_t o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                o[j] = (uint32_t)t16[(chunk * 8 + 2 * j) * 66 + nl] | ((uint32_t)t16[(chunk * 8 + 2 * j + 1) * 66 + nl] << 16);
-            *reinterpret_cast<uint4 *>(a2 + (long long)n * M + m) = make_uint4(o[0], o[1], o[2], o[3]);
-        }
-    }
-}
-
-// packed codes [rows x K] -> ct [K x rows] bfloat16 grid values c = 2k - (2^b - 1).
-// Tiles of 64 rows x 128 columns, 256 threads: a thread expands whole 32-bit code words into
-// shared memory, then the tile leaves transposed in 16-byte pieces (rows is a multiple of 8).
+// Packed level indices and per-row scales -> dequantised values bf16(scale[r] * c) [rows x K], dense.
+// One thread converts 8 consecutive elements (one 16-byte store; K % 32 == 0 keeps them in one row).
 template <int CB>
 __global__ void __launch_bounds__(256)
-codes_to_bf16_t_kernel(const uint8_t *__restrict__ codes, int bits, int rows, int K, uint16_t *__restrict__ ct) {
-    __shared__ __align__(16) uint16_t tile[128][72];           // [k][row], pitch 144 bytes
+dequant_codes_kernel(const uint8_t *__restrict__ codes0, const float *__restrict__ scales0, uint16_t *__restrict__ out0,
+                     long long n_oct0, const uint8_t *__restrict__ codes1, const float *__restrict__ scales1,
+                     uint16_t *__restrict__ out1, long long n_oct1, int bits, int K) {
     pdl_launch_dependents();
     pdl_wait();
-    constexpr int PER = 32 / CB;                               // codes per word
-    constexpr int WPR = 128 / PER;                             // words per tile row
+    long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_oct0 + n_oct1) return;
+    const bool second = t >= n_oct0;                         // up to two tensors per launch
+    if (second) t -= n_oct0;
+    const uint8_t *codes = second ? codes1 : codes0;
+    const float *scales = second ? scales1 : scales0;
+    uint16_t *out = second ? out1 : out0;
     const int L1 = (1 << bits) - 1;
-    const int r0 = blockIdx.y * 64, k0 = blockIdx.x * 128;
-    const int t = threadIdx.x;
-    const long long row_words = (long long)K * CB / 32;
+    const float sc = __ldg(scales + t / (K / 8));
+    const uint32_t *c32 = reinterpret_cast<const uint32_t *>(codes);
+    uint32_t lo, hi = 0;                                     // the 8 * CB bits of this thread's levels
+    if constexpr (CB == 8) { lo = __ldg(c32 + 2 * t); hi = __ldg(c32 + 2 * t + 1); }
+    else if constexpr (CB == 4) lo = __ldg(c32 + t);
+    else if constexpr (CB == 2) lo = (__ldg(c32 + (t >> 1)) >> (16 * (int)(t & 1))) & 0xFFFFu;
+    else lo = (__ldg(c32 + (t >> 2)) >> (8 * (int)(t & 3))) & 0xFFu;
+    uint32_t o[4];
 #pragma unroll
-    for (int i = 0; i < (64 * WPR) / 256; ++i) {
-        const int w = t + 256 * i;
-        const int rl = w & 63, wl = w >> 6;                    // consecutive lanes: consecutive rows (conflict-free tile writes)
-        const int r = r0 + rl, k = k0 + wl * PER;
-        uint32_t word = 0;
-        const bool ok = r < rows && k < K;
-        if (ok) word = __ldg(reinterpret_cast<const uint32_t *>(codes) + r * row_words + (k0 / PER) + wl);
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int lev = (word >> (j * CB)) & ((1 << CB) - 1);
-            tile[wl * PER + j][rl] = ok ? bf16_bits((float)(2 * lev - L1)) : (uint16_t)0;    // |c| <= 255: exact
+    for (int j = 0; j < 4; ++j) {
+        int k0, k1;
+        if constexpr (CB == 8) {
+            const uint32_t w = j < 2 ? lo : hi;
+            k0 = (int)((w >> (16 * (j & 1))) & 0xFFu);
+            k1 = (int)((w >> (16 * (j & 1) + 8)) & 0xFFu);
+        } else {
+            k0 = (int)((lo >> (2 * j * CB)) & ((1u << CB) - 1u));
+            k1 = (int)((lo >> ((2 * j + 1) * CB)) & ((1u << CB) - 1u));
         }
+        o[j] = (uint32_t)bf16_bits(sc * (float)(2 * k0 - L1)) | ((uint32_t)bf16_bits(sc * (float)(2 * k1 - L1)) << 16);
     }
-    __syncthreads();
-    const int chunk = t & 7;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int kl = (t >> 3) + 32 * i;
-        const int k = k0 + kl, r = r0 + chunk * 8;
-        if (k < K && r < rows)
-            *reinterpret_cast<uint4 *>(ct + (long long)k * rows + r) = *reinterpret_cast<const uint4 *>(&tile[kl][chunk * 8]);
-    }
+    *reinterpret_cast<uint4 *>(out + t * 8) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // Inverse orthonormal block Hadamard transform of every row of d [rows x cols] (binary32, dense),
@@ -214,8 +163,8 @@ iht_rows_kernel(const void *__restrict__ d, int in_dtype, long long ld_in, long 
 }
 
 struct BwdWorkspace {
-    uint16_t *a1, *a2, *cwt, *cxt;
-    float *d1, *d2;
+    uint16_t *wh, *xh;      // dequantised operands [N x K], [M x K]
+    float *d1, *d2;         // masked products when the inverse transform is a separate kernel
     size_t bytes;
 };
 BwdWorkspace carve_bwd(void *base, int64_t M, int64_t N, int64_t K) {
@@ -223,10 +172,8 @@ BwdWorkspace carve_bwd(void *base, int64_t M, int64_t N, int64_t K) {
     uint8_t *b = reinterpret_cast<uint8_t *>(base);
     size_t off = 0;
     auto take = [&](size_t n) { uint8_t *p = b + off; off += align_up(n, 256); return p; };
-    w.a1 = reinterpret_cast<uint16_t *>(take((size_t)M * N * 2));
-    w.a2 = reinterpret_cast<uint16_t *>(take((size_t)M * N * 2));
-    w.cwt = reinterpret_cast<uint16_t *>(take((size_t)K * N * 2));
-    w.cxt = reinterpret_cast<uint16_t *>(take((size_t)K * M * 2));
+    w.wh = reinterpret_cast<uint16_t *>(take((size_t)N * K * 2));
+    w.xh = reinterpret_cast<uint16_t *>(take((size_t)M * K * 2));
     w.d1 = reinterpret_cast<float *>(take((size_t)M * K * 4));
     w.d2 = reinterpret_cast<float *>(take((size_t)N * K * 4));
     w.bytes = off;
@@ -292,7 +239,7 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
         return QUEST_ERR_HAD_BLOCK;
     if (out_dtype != QUEST_F32 && out_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
     auto al = [](const void *p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; };
-    if (!al(dy, 16) || !al(mx, 16) || !al(mw, 16) || !al(sw, 16) || !al(xq, 4) || !al(wq, 4) || (dx && !al(dx, 16)) ||
+    if (!al(dy, 16) || !al(mx, 16) || !al(mw, 16) || !al(sw, 4) || !al(sx, 4) || !al(xq, 4) || !al(wq, 4) || (dx && !al(dx, 16)) ||
         (dw && !al(dw, 16)))
         return QUEST_ERR_ALIGN;
     if (!workspace || !al(workspace, 256) || workspace_bytes < quest_bwd_workspace_bytes(M, N, K))
@@ -306,43 +253,38 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
         Stage(int id, cudaStream_t s_) : h(stage_begin(id, s_)) {}
         ~Stage() { stage_end(h); }
     };
-    Stage *prep = new Stage(QUEST_STAGE_UNPACK, st);   // operand preparation of the whole call up to the first product
-    cudaError_t e = launch_pdl(scale_dy_kernel, dim3((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64)), dim3(256), 0, st, 1,
-                               reinterpret_cast<const uint16_t *>(dy), sx, sw, (int)M, (int)N, ws.a1, ws.a2);
-    if (e != cudaSuccess) { delete prep; return cuda_fail(e); }
-    auto codes_t = [&](const uint8_t *codes, int64_t rows, uint16_t *ct) -> cudaError_t {
-        const dim3 grid((unsigned)((K + 127) / 128), (unsigned)((rows + 63) / 64));
+    {
+        // both dequantised operands in one launch, then the two products back to back
+        Stage prep(QUEST_STAGE_UNPACK, st);
+        const long long n0 = dx ? (long long)N * (K / 8) : 0, n1 = dw ? (long long)M * (K / 8) : 0;
+        const dim3 grid((unsigned)((n0 + n1 + 255) / 256));
+        cudaError_t e;
         switch (container_bits(bits)) {
-            case 1: return launch_pdl(codes_to_bf16_t_kernel<1>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
-            case 2: return launch_pdl(codes_to_bf16_t_kernel<2>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
-            case 4: return launch_pdl(codes_to_bf16_t_kernel<4>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
-            default: return launch_pdl(codes_to_bf16_t_kernel<8>, grid, dim3(256), 0, st, 1, codes, bits, (int)rows, (int)K, ct);
+            case 1: e = launch_pdl(dequant_codes_kernel<1>, grid, dim3(256), 0, st, 1, wq, sw, ws.wh, n0, xq, sx, ws.xh, n1, bits, (int)K); break;
+            case 2: e = launch_pdl(dequant_codes_kernel<2>, grid, dim3(256), 0, st, 1, wq, sw, ws.wh, n0, xq, sx, ws.xh, n1, bits, (int)K); break;
+            case 4: e = launch_pdl(dequant_codes_kernel<4>, grid, dim3(256), 0, st, 1, wq, sw, ws.wh, n0, xq, sx, ws.xh, n1, bits, (int)K); break;
+            default: e = launch_pdl(dequant_codes_kernel<8>, grid, dim3(256), 0, st, 1, wq, sw, ws.wh, n0, xq, sx, ws.xh, n1, bits, (int)K); break;
         }
-    };
-    if (dx) {
-        e = codes_t(wq, N, ws.cwt);
-        if (prep) { delete prep; prep = nullptr; }
         if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (dx) {
         Stage gemm_stage(QUEST_STAGE_GEMM, st);
-        // line 2 and the mask of line 3: d1[m][k] = M_x[m][k] * sum_n a1[m][n] cwt[k][n]
+        // line 2 and the mask of line 3: d1[m][k] = M_x[m][k] * sum_n dy[m][n] wq_h[n][k]
         // (blocks of 128: the inverse transform is fused into the contraction's epilogue)
         if (had_block == 128 && M > 128 && K > 128) {
-            if ((s = launch_gemm_bf16_masked(ws.a1, ws.cwt, M, K, N, mx, dx, out_dtype, true, st))) return s;
+            if ((s = launch_gemm_bf16_masked(dy, ws.wh, M, K, N, mx, dx, out_dtype, true, 1, st))) return s;
         } else {
-            if ((s = launch_gemm_bf16_masked(ws.a1, ws.cwt, M, K, N, mx, ws.d1, QUEST_F32, false, st))) return s;
+            if ((s = launch_gemm_bf16_masked(dy, ws.wh, M, K, N, mx, ws.d1, QUEST_F32, false, 1, st))) return s;
             if ((s = launch_iht(ws.d1, M, K, had_block, dx, out_dtype, K, st))) return s;
         }
     }
     if (dw) {
-        e = codes_t(xq, M, ws.cxt);
-        if (prep) { delete prep; prep = nullptr; }
-        if (e != cudaSuccess) return cuda_fail(e);
         Stage gemm_stage(QUEST_STAGE_GEMM, st);
-        // line 4 and the mask of line 5: d2[n][k] = M_w[n][k] * sum_m a2[n][m] cxt[k][m]
+        // line 4 and the mask of line 5: d2[n][k] = M_w[n][k] * sum_m dy[m][n] xq_h[m][k]
         if (had_block == 128 && N > 128 && K > 128) {
-            if ((s = launch_gemm_bf16_masked(ws.a2, ws.cxt, N, K, M, mw, dw, out_dtype, true, st))) return s;
+            if ((s = launch_gemm_bf16_masked(dy, ws.xh, N, K, M, mw, dw, out_dtype, true, 2, st))) return s;
         } else {
-            if ((s = launch_gemm_bf16_masked(ws.a2, ws.cxt, N, K, M, mw, ws.d2, QUEST_F32, false, st))) return s;
+            if ((s = launch_gemm_bf16_masked(dy, ws.xh, N, K, M, mw, ws.d2, QUEST_F32, false, 2, st))) return s;
             if ((s = launch_iht(ws.d2, N, K, had_block, dw, out_dtype, K, st))) return s;
         }
     }

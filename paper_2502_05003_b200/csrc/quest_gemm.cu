@@ -129,6 +129,19 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;                                // layout: SWIZZLE_128B, bits [61,64)
     return d;
 }
+// The same for an MN-major 16-bit operand as TMA lays it out: rows of 128 bytes hold 64 consecutive
+// elements of the M (or N) dimension for one k; eight consecutive k form a 1024-byte swizzle atom;
+// the next eight k follow 1024 bytes later (stride byte offset), the next 64 elements of M / N
+// 8192 bytes later (leading byte offset: one 64 x 64 chunk).
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)(8192 >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
 // Instruction descriptor for kind::i8: D = s32, A = B = signed 8-bit, both K-major.
 __host__ __device__ constexpr uint32_t make_idesc_i8(int m, int n) {
     return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
@@ -287,7 +300,10 @@ struct SmemLayout {
 // kind::mxf4 with unit block scales; the binary32 accumulators hold sum v_x v_w exactly (multiples of
 // 1/4 below 2^22), reported as acc4 = 4 * sum; tensor memory holds one accumulator buffer of 256
 // columns (or two of 128) and the scale bytes.
-template <int BN, int MODE, bool TWO, bool YT>
+// OPL (bfloat16 modes only): 0 = both operands K-major; 1 = B MN-major (its memory rows run along the
+// contraction); 2 = A and B MN-major.  The backward pass uses 1 and 2 to read dy and the dequantised
+// operands as they lie in memory, without transposed copies.
+template <int BN, int MODE, bool TWO, bool YT, int OPL = 0>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
@@ -300,6 +316,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr int NBUF = (MX && BN == 256) ? 1 : 2;   // accumulator buffers in tensor memory
     constexpr uint32_t SF_COL = 256;              // MX: 32 columns of scale bytes after the accumulators
     constexpr bool IHT128 = MODE == 3;
+    constexpr bool AMN = OPL == 2, BMN = OPL >= 1;
+    static_assert(OPL == 0 || MODE == 2 || MODE == 3, "MN-major operands: bfloat16 backward modes only");
     static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
     constexpr int STAGES = L::NSTAGES;
     constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
@@ -391,16 +409,42 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!ok) break;
                     const uint32_t fb = smem_u32(&full_bar[stage]);
                     uint8_t *sa = smem + stage * L::STAGE_BYTES;
+                    // K-major: one box of 128 bytes of K x rows.  MN-major: 64 x 64 chunks (128 bytes of the
+                    // M / N dimension x 64 k), 8192 bytes each, in the order of the M / N dimension.
                     if constexpr (TWO) {
                         // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
                         if (leader) mbar_expect_tx(fb, 2 * L::STAGE_BYTES);
                         const uint32_t lfb = mapa_shared(fb, 0);
-                        tma_load_2d_pair(smem_u32(sa), &tmA, kb * BK, m0, lfb);
-                        tma_load_2d_pair(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, lfb);
+                        if constexpr (AMN) {
+#pragma unroll
+                            for (int c = 0; c < BM / 64; ++c)
+                                tma_load_2d_pair(smem_u32(sa + c * 8192), &tmA, (m0 + 64 * c) * 2, kb * 64, lfb);
+                        } else {
+                            tma_load_2d_pair(smem_u32(sa), &tmA, kb * BK, m0, lfb);
+                        }
+                        if constexpr (BMN) {
+#pragma unroll
+                            for (int c = 0; c < L::B_ROWS / 64; ++c)
+                                tma_load_2d_pair(smem_u32(sa + L::A_BYTES + c * 8192), &tmB, (n0 + 64 * c) * 2, kb * 64, lfb);
+                        } else {
+                            tma_load_2d_pair(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, lfb);
+                        }
                     } else {
                         mbar_expect_tx(fb, L::STAGE_BYTES);
-                        tma_load_2d(smem_u32(sa), &tmA, kb * BK, m0, fb);
-                        tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
+                        if constexpr (AMN) {
+#pragma unroll
+                            for (int c = 0; c < BM / 64; ++c)
+                                tma_load_2d(smem_u32(sa + c * 8192), &tmA, (m0 + 64 * c) * 2, kb * 64, fb);
+                        } else {
+                            tma_load_2d(smem_u32(sa), &tmA, kb * BK, m0, fb);
+                        }
+                        if constexpr (BMN) {
+#pragma unroll
+                            for (int c = 0; c < L::B_ROWS / 64; ++c)
+                                tma_load_2d(smem_u32(sa + L::A_BYTES + c * 8192), &tmB, (n0 + 64 * c) * 2, kb * 64, fb);
+                        } else {
+                            tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
+                        }
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -416,7 +460,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0 && leader) {
-            constexpr uint32_t idesc = MX ? make_idesc_mxf4(TILE_M, BN) : F16 ? make_idesc_bf16(TILE_M, BN) : make_idesc_i8(TILE_M, BN);
+            constexpr uint32_t idesc = MX ? make_idesc_mxf4(TILE_M, BN)
+                                          : F16 ? (make_idesc_bf16(TILE_M, BN) | (AMN ? 1u << 15 : 0u) | (BMN ? 1u << 16 : 0u))
+                                                : make_idesc_i8(TILE_M, BN);
             int stage = 0;
             uint32_t phase = 0;
             int t = 0;
@@ -433,13 +479,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + stage * L::STAGE_BYTES);
-                    const uint64_t a_desc = make_smem_desc(sa);
-                    const uint64_t b_desc = make_smem_desc(sa + L::A_BYTES);
+                    const uint64_t a_desc = AMN ? make_smem_desc_mn(sa) : make_smem_desc(sa);
+                    const uint64_t b_desc = BMN ? make_smem_desc_mn(sa + L::A_BYTES) : make_smem_desc(sa + L::A_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-                        // advance along K inside the 128-byte swizzle row: +32 bytes = +2 in 16-byte units
-                        const uint64_t ad = a_desc + (uint64_t)(kk * (UMMA_K >> 4));
-                        const uint64_t bd = b_desc + (uint64_t)(kk * (UMMA_K >> 4));
+                        // advance along K: K-major +32 bytes inside the 128-byte swizzle row (+2 in 16-byte units);
+                        // MN-major 16 k = two 1024-byte atoms further (+128)
+                        const uint64_t ad = a_desc + (uint64_t)(kk * (AMN ? 128 : (UMMA_K >> 4)));
+                        const uint64_t bd = b_desc + (uint64_t)(kk * (BMN ? 128 : (UMMA_K >> 4)));
                         const uint32_t accum = (kb | kk) != 0 ? 1u : 0u;
                         if constexpr (MX) {       // 32 bytes of K = 64 E2M1 per instruction
                             if constexpr (TWO) umma_mxf4_pair(d_tmem, ad, bd, idesc, accum, tmem_base + SF_COL, tmem_base + SF_COL + 16);
@@ -847,13 +894,13 @@ int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes
     return QUEST_OK;
 }
 
-template <int BN, int MODE, bool TWO, bool YT>
+template <int BN, int MODE, bool TWO, bool YT, int OPL = 0>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
                    cudaStream_t st) {
     using L = SmemLayout<BN, TWO>;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, MODE, TWO, YT>,
+        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, MODE, TWO, YT, OPL>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
         attr_done = true;
@@ -870,7 +917,7 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
     } else {
         grid = tiles < sms ? tiles : sms;
     }
-    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
+    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT, OPL>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
                                TWO ? 2 : 1, tmA, tmB, tmY, p);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
@@ -977,12 +1024,15 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
 #undef QUEST_GEMM
 }
 
-// Backward-pass contraction (Algorithm 2, lines 2 and 4): out[i][j] = mask[i][j] * sum_k a[i][k] b[j][k]
-// with bfloat16 operands a [I x Kc], b [J x Kc] (both dense, Kc contiguous) and binary32 output [I x J].
+// Backward-pass contraction (Algorithm 2, lines 2 and 4): out[i][j] = mask[i][j] * sum_k A(i, k) B(j, k) with
+// bfloat16 operands and binary32 output [I x J].  `opl` says how the operands lie in memory:
+//   0: a [I x Kc], b [J x Kc], the contraction index contiguous (K-major);
+//   1: a [I x Kc] K-major, b [Kc x J] (memory rows run along the contraction: MN-major);
+//   2: a [Kc x I] and b [Kc x J], both MN-major.
 // With fuse_iht128 (J % 128 == 0, I > 128, J > 128) the epilogue also applies the inverse Hadamard
 // transform on blocks of 128 columns and stores out_dtype; otherwise out is binary32.
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
-                            const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st) {
+                            const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, int opl, cudaStream_t st) {
     if (I == 0 || J == 0) return QUEST_OK;
     GemmParams p;
     p.M = (int)I; p.N = (int)J; p.K = (int)(2 * Kc);
@@ -995,20 +1045,29 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     const bool wide = J > 128;
     const bool pair = wide && I > 128;
     CUtensorMap tmA, tmB, tmY;
-    int s = make_operand_map(&tmA, reinterpret_cast<const int8_t *>(a), I, 2 * Kc, BM);
+    int s;
+    // MN-major: the tensor is [Kc rows x I (or J) elements]; a box is 128 bytes of a row x 64 rows
+    if (opl == 2) s = make_operand_map(&tmA, reinterpret_cast<const int8_t *>(a), Kc, 2 * I, 64);
+    else s = make_operand_map(&tmA, reinterpret_cast<const int8_t *>(a), I, 2 * Kc, BM);
     if (s) return s;
-    s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(b), J, 2 * Kc, pair ? 128 : wide ? 256 : 128);
+    if (opl >= 1) s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(b), Kc, 2 * J, 64);
+    else s = make_operand_map(&tmB, reinterpret_cast<const int8_t *>(b), J, 2 * Kc, pair ? 128 : wide ? 256 : 128);
     if (s) return s;
     s = make_output_map(&tmY, out, I, J * esz, J * esz);
     if (s) return s;
+#define QUEST_GEMM_BWD(BNV, MODEV, TWOV)                                                  \
+    (opl == 2 ? launch_gemm_bn<BNV, MODEV, TWOV, true, 2>(tmA, tmB, tmY, p, st)           \
+              : opl == 1 ? launch_gemm_bn<BNV, MODEV, TWOV, true, 1>(tmA, tmB, tmY, p, st) \
+                         : launch_gemm_bn<BNV, MODEV, TWOV, true, 0>(tmA, tmB, tmY, p, st))
     if (fuse_iht128) {
         if (!pair || J % 128 != 0) return QUEST_ERR_SHAPE;
-        return launch_gemm_bn<256, 3, true, true>(tmA, tmB, tmY, p, st);
+        return QUEST_GEMM_BWD(256, 3, true);
     }
     if (out_dtype != QUEST_F32) return QUEST_ERR_DTYPE;
-    if (pair) return launch_gemm_bn<256, 2, true, true>(tmA, tmB, tmY, p, st);
-    if (wide) return launch_gemm_bn<256, 2, false, true>(tmA, tmB, tmY, p, st);
-    return launch_gemm_bn<128, 2, false, true>(tmA, tmB, tmY, p, st);
+    if (pair) return QUEST_GEMM_BWD(256, 2, true);
+    if (wide) return QUEST_GEMM_BWD(256, 2, false);
+    return QUEST_GEMM_BWD(128, 2, false);
+#undef QUEST_GEMM_BWD
 }
 
 // Contraction of E2M1 nibble operands xq [M x K/2], wq [N x K/2] on the FP4 tensor-core path:

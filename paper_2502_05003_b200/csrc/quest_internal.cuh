@@ -127,8 +127,9 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
 void *stage_begin(int id, cudaStream_t st);
 void stage_end(void *scope);
 
+// opl: 0 both operands K-major ([rows x Kc]); 1 b MN-major ([Kc x J]); 2 a and b MN-major ([Kc x I], [Kc x J]).
 int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, int64_t Kc,
-                            const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, cudaStream_t st);
+                            const uint8_t *mask, void *out, int out_dtype, bool fuse_iht128, int opl, cudaStream_t st);
 
 // Contraction of E2M1 nibble operands (tcgen05 kind::mxf4, unit block scales): acc = acc_mul * sum v_x v_w
 // (int32, exact), y = sx sw sum v_x v_w.  xq, wq 16-byte aligned, K % 32 == 0.  Serves the FP4 grid
