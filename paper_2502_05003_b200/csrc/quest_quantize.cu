@@ -192,8 +192,8 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // applied by the caller), RMS, projection, trust test, packing and stores for the E elements this
 // thread holds.  GFULL: had_block >= E, so every in-register stage runs.  FAST: the common case
 // fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
-// one warp, every output requested, no row sums, trust_factor >= 1 -- so that no per-row branch or
-// loop remains.
+// one warp, codes, scales and mask requested (the GEMM operand is optional), no row sums,
+// trust_factor >= 1 -- so that no per-row loop and only one uniform branch remain.
 template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
@@ -449,13 +449,13 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
             if constexpr (GRID == GRID_UNIFORM) {              // the FP4 codes are themselves the tensor-core operand
             if constexpr (CB <= 2) {
                 // one- and two-bit grids: E2M1 nibbles for the FP4 tensor-core path, 16 bytes per 32 elements
-                if (FAST || tn.op8) {
+                if (tn.op8) {                                   // uniform over the CTA
                     uint32_t o[4];
                     e2m1_operand_from_code_words<CB>(w, o);
                     *reinterpret_cast<uint4 *>(tn.op8 + row * (long long)(cols >> 1) + (long long)tr * (E / 2) + g32 * 16) =
                         make_uint4(o[0], o[1], o[2], o[3]);
                 }
-            } else if (FAST || tn.op8) {
+            } else if (tn.op8) {
                 uint32_t o[8];
                 operand_from_code_words<CB>(w, a.bits, o);
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
@@ -758,7 +758,7 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 bool fast = had_block == 128 && S >= 32 && bits < 8 && trust_factor >= 1.0f;
                 for (int j = 0; j < 2; ++j) {
                     const QuantTensor &t = a.t[j];
-                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && t.op8 && !t.rowsum && !t.rot && !t.cbf)) fast = false;
+                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && !t.rowsum && !t.rot && !t.cbf)) fast = false;
                 }
                 if (grid_kind == GRID_FP4) {
                     // the FP4 codes are the GEMM operand themselves: the specialised path wants codes, scales, mask
