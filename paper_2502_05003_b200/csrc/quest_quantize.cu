@@ -194,7 +194,7 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
 // one warp, codes, scales and mask requested (the GEMM operand is optional), no row sums,
 // trust_factor >= 1 -- so that no per-row loop and only one uniform branch remain.
-template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM>
+template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
                                                      int s_start) {
@@ -220,7 +220,9 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
 #pragma unroll
         for (int i = 0; i < H; ++i) v[i] = __ffma2_rn(v[i], sgn, x2[i * nthreads + pt]);
     }
-    if constexpr (FAST) {
+    if constexpr (XDONE) {
+        // the caller has applied every stride that pairs this thread with another one
+    } else if constexpr (FAST) {
         if constexpr (E == 32) {                               // stride 32: partner is the neighbouring lane
             const float sg = (lane & 1) ? -1.0f : 1.0f;
             const float2 sgn = make_float2(sg, sg);
@@ -630,6 +632,171 @@ quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, in
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
+// Wide rotation blocks (had_block = 1024, 2048 or 4096, bfloat16 rows): the five largest strides are
+// made thread-local by a change of data layout instead of five rounds of warp shuffles.  A block of
+// g = 32 G elements belongs to G threads.  Phase A: thread p of the block takes the 32 elements
+// p + G j (j = 0..31) from the raw row in shared memory, so the strides g/2 .. g/32 pair elements
+// it already holds (one in-register 32-point butterfly, largest stride first).  The result goes
+// back to shared memory in row order (binary32, 16 bytes of padding per 32 elements).  Phase B:
+// every thread reads its 32 contiguous elements; the one or two strides left between g/64 and 32
+// pair it with threads tr ^ 1, tr ^ 2, whose elements it reads from the same buffer; the strides
+// below 32 and everything after the rotation are the common tail.  The order of the butterfly stages
+// and every operand of every addition are those of the other kernels: the results are identical.
+__device__ __forceinline__ void butterfly32_in_registers(float2 (&v)[16]) {
+    const float2 neg1 = make_float2(-1.0f, -1.0f);
+#pragma unroll
+    for (int s2 = 8; s2 >= 1; s2 >>= 1) {                      // element strides 16 .. 2
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if ((i & s2) == 0) {
+                const float2 p = v[i], q = v[i + s2];
+                v[i] = __fadd2_rn(p, q);
+                v[i + s2] = __ffma2_rn(q, neg1, p);
+            }
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {                             // element stride 1
+        const float p = v[i].x, q = v[i].y;
+        v[i] = make_float2(__fadd_rn(p, q), __fsub_rn(p, q));
+    }
+}
+
+template <int CB, bool FAST, int GRID = GRID_UNIFORM>
+__global__ void __launch_bounds__(256, 3)
+quantize_wide_kernel(const __grid_constant__ QuantArgs a, int total_groups, int exchange_bytes) {
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int cols = a.cols, S = a.S, R = a.R;
+    const int G = a.had_block >> 5;                            // threads per rotation block: 32, 64 or 128
+    const int gshift = 31 - __clz(G);
+    float *xsm = reinterpret_cast<float *>(smem_raw);
+    float *tbuf = reinterpret_cast<float *>(smem_raw + exchange_bytes);
+    const int trow_words = cols + (cols >> 3);                 // 36 words per 32 elements
+    uint8_t *raw = reinterpret_cast<uint8_t *>(tbuf + (size_t)R * trow_words);
+    const int tid = threadIdx.x;
+    const int r_local = tid / S;
+    const int tr = tid - r_local * S;
+    const int p = tr & (G - 1);
+    const int blk_base = (tr >> gshift) * a.had_block;         // first element of this thread's block
+
+    auto locate = [&](int grp, int &which, long long &row) {
+        which = grp >= a.blocks0 ? 1 : 0;
+        row = (long long)(which ? grp - a.blocks0 : grp) * R + r_local;
+    };
+    auto prefetch = [&](int grp, int buf) {
+        if (grp < total_groups) {
+            int which;
+            long long row;
+            locate(grp, which, row);
+            const QuantTensor &tn = a.t[which];
+            const bool live = row < tn.rows;
+            const uint8_t *src = live ? reinterpret_cast<const uint8_t *>(tn.x) + (row * tn.ld + (long long)tr * 32) * 2
+                                      : reinterpret_cast<const uint8_t *>(tn.x);
+            const uint32_t nbytes = live ? 16u : 0u, step = live ? 16u : 0u;
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(raw + ((size_t)(buf * R + r_local) * cols + (size_t)tr * 32) * 2);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + q * 16), "l"(src + q * step), "r"(nbytes)
+                             : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    int buf = 0;
+    prefetch((int)blockIdx.x, 0);
+    for (int grp = (int)blockIdx.x; grp < total_groups; grp += (int)gridDim.x, buf ^= 1) {
+        prefetch(grp + (int)gridDim.x, buf ^ 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        __syncthreads();                                       // the whole row has landed; last round's readers are done
+        int which;
+        long long row;
+        locate(grp, which, row);
+        const QuantTensor &tn = a.t[which];
+        const bool active = row < tn.rows;
+        float2 v[16];
+        {   // phase A: elements p + G j of this thread's block, then strides g/2 .. g/32 in registers
+            const uint16_t *rrow = reinterpret_cast<const uint16_t *>(raw + (size_t)(buf * R + r_local) * cols * 2) + blk_base + p;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                v[j] = make_float2(__uint_as_float((uint32_t)rrow[(2 * j) << gshift] << 16),
+                                   __uint_as_float((uint32_t)rrow[(2 * j + 1) << gshift] << 16));
+            butterfly32_in_registers(v);
+            float *trow = tbuf + (size_t)r_local * trow_words;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int i0 = blk_base + p + ((2 * j) << gshift), i1 = blk_base + p + ((2 * j + 1) << gshift);
+                trow[i0 + ((i0 >> 5) << 2)] = v[j].x;
+                trow[i1 + ((i1 >> 5) << 2)] = v[j].y;
+            }
+        }
+        __syncthreads();
+        {   // phase B: 32 contiguous elements; strides g/64 .. 32 against the partner threads' elements
+            const float *trow = tbuf + (size_t)r_local * trow_words;
+            const float4 *own = reinterpret_cast<const float4 *>(trow + tr * 36);
+            if (G == 32) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 o = own[q];
+                    v[2 * q] = make_float2(o.x, o.y);
+                    v[2 * q + 1] = make_float2(o.z, o.w);
+                }
+            } else if (G == 64) {
+                const float4 *p1 = reinterpret_cast<const float4 *>(trow + (tr ^ 1) * 36);
+                const float s1 = (tr & 1) ? -1.0f : 1.0f;
+                const float2 sg1 = make_float2(s1, s1);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 o = own[q], b = p1[q];
+                    v[2 * q] = __ffma2_rn(make_float2(o.x, o.y), sg1, make_float2(b.x, b.y));
+                    v[2 * q + 1] = __ffma2_rn(make_float2(o.z, o.w), sg1, make_float2(b.z, b.w));
+                }
+            } else {
+                const float4 *p1 = reinterpret_cast<const float4 *>(trow + (tr ^ 1) * 36);
+                const float4 *p2 = reinterpret_cast<const float4 *>(trow + (tr ^ 2) * 36);
+                const float4 *p3 = reinterpret_cast<const float4 *>(trow + (tr ^ 3) * 36);
+                const float s1 = (tr & 1) ? -1.0f : 1.0f, s2 = (tr & 2) ? -1.0f : 1.0f;
+                const float2 sg1 = make_float2(s1, s1), sg2 = make_float2(s2, s2);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 o = own[q], b1 = p1[q], b2 = p2[q], b3 = p3[q];
+                    // stride 64: this thread with tr ^ 2, and thread tr ^ 1 with tr ^ 3 (same side, same sign)
+                    const float2 u0 = __ffma2_rn(make_float2(o.x, o.y), sg2, make_float2(b2.x, b2.y));
+                    const float2 u1 = __ffma2_rn(make_float2(o.z, o.w), sg2, make_float2(b2.z, b2.w));
+                    const float2 w0 = __ffma2_rn(make_float2(b1.x, b1.y), sg2, make_float2(b3.x, b3.y));
+                    const float2 w1 = __ffma2_rn(make_float2(b1.z, b1.w), sg2, make_float2(b3.z, b3.w));
+                    // stride 32: this thread's result with that of thread tr ^ 1
+                    v[2 * q] = __ffma2_rn(u0, sg1, w0);
+                    v[2 * q + 1] = __ffma2_rn(u1, sg1, w1);
+                }
+            }
+        }
+        rotate_project_store<CB, 32, true, FAST, GRID, true>(v, a, tn, active, row, tr, r_local, xsm, 16);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+template <int GRID, bool FAST>
+static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                               int total_groups, int exchange_bytes) {
+#define QUEST_LAUNCH(CBV)                                                                                   \
+    do {                                                                                                    \
+        cudaError_t e_ = cudaFuncSetAttribute(quantize_wide_kernel<CBV, FAST, GRID>,                        \
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);     \
+        if (e_ != cudaSuccess) return e_;                                                                   \
+        return launch_pdl(quantize_wide_kernel<CBV, FAST, GRID>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
+                          total_groups, exchange_bytes);                                                    \
+    } while (0)
+    if (GRID == GRID_FP4) QUEST_LAUNCH(4);
+    switch (cb) {
+        case 1: QUEST_LAUNCH(1);
+        case 2: QUEST_LAUNCH(2);
+        case 4: QUEST_LAUNCH(4);
+        default: QUEST_LAUNCH(8);
+    }
+#undef QUEST_LAUNCH
+}
+
 template <bool BF16, int E>
 static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
@@ -745,6 +912,33 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 else
                     e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 32>(grid, threads, smem, st, a)
                                             : launch_rows_fp4<false, 32>(grid, threads, smem, st, a);
+            } else if (streaming && E == 32 && S == T && S <= 256 &&
+                       (had_block == 1024 || had_block == 2048 || had_block == 4096)) {
+                // wide rotation blocks: layout-change kernel (persistent, double-buffered raw rows)
+                const int exchange = (int)((sizeof(float) * (size_t)warps + 15) / 16 * 16);
+                const size_t smem2 = (size_t)exchange + (size_t)R * (cols + cols / 8) * 4 + 2 * (size_t)R * cols * 2;
+                int dev = 0, sms = 148;
+                cudaGetDevice(&dev);
+                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+                int per_sm = (int)((220 * 1024) / (smem2 + 1024));
+                const int by_threads = 1024 / threads;
+                if (per_sm > by_threads) per_sm = by_threads;
+                if (per_sm < 1) per_sm = 1;
+                const int total = nb[0] + nb[1];
+                const int g = total < sms * per_sm ? total : sms * per_sm;
+                // the specialised tail (codes, scales and masks requested, trust_factor >= 1, below 8 bits)
+                bool fastw = bits < 8 && trust_factor >= 1.0f;
+                for (int j = 0; j < 2; ++j) {
+                    const QuantTensor &t = a.t[j];
+                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && !t.rowsum && !t.rot && !t.cbf)) fastw = false;
+                    if (t.rows > 0 && grid_kind == GRID_FP4 && t.op8) fastw = false;
+                }
+                if (grid_kind == GRID_FP4)
+                    e = fastw ? launch_wide<GRID_FP4, true>(cb, g, threads, smem2, st, a, total, exchange)
+                              : launch_wide<GRID_FP4, false>(cb, g, threads, smem2, st, a, total, exchange);
+                else
+                    e = fastw ? launch_wide<GRID_UNIFORM, true>(cb, g, threads, smem2, st, a, total, exchange)
+                              : launch_wide<GRID_UNIFORM, false>(cb, g, threads, smem2, st, a, total, exchange);
             } else if (streaming) {
                 // persistent streaming kernel: as many CTAs as fit on the device, each looping over groups
                 const int exchange = (int)((smem + 15) / 16 * 16);

@@ -53,7 +53,8 @@ def rows_of(kind, rows, cols, seed, bf16):
 
 @pytest.mark.parametrize("bits", [1, 2, 3, 4, 5, 8])
 @pytest.mark.parametrize("g,cols", [(1, 64), (8, 256), (32, 96), (64, 640), (128, 128), (128, 2048), (128, 5504),
-                                    (256, 768), (512, 512), (1024, 3072), (2048, 2048), (4096, 4096)])
+                                    (256, 768), (512, 512), (1024, 1024), (1024, 3072), (2048, 2048), (2048, 4096),
+                                    (4096, 4096)])
 def test_bf16_rows(bits, g, cols):
     check(rows_of("student", 67, cols, bits * 100 + g, True), bits, g)
 
