@@ -192,8 +192,9 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // applied by the caller), RMS, projection, trust test, packing and stores for the E elements this
 // thread holds.  GFULL: had_block >= E, so every in-register stage runs.  FAST: the common case
 // fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
-// one warp, codes, scales and mask requested (the GEMM operand is optional), no row sums,
-// trust_factor >= 1 -- so that no per-row loop and only one uniform branch remain.
+// one warp, codes, scales and mask requested (the GEMM operand and the bfloat16 outputs of the
+// weight-only variant are optional; a tensor may also ask for the rotation alone), no row sums,
+// trust_factor >= 1 -- so that no per-row loop and only a few uniform branches remain.
 template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
@@ -273,7 +274,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
     }
 
     // ---- the rotation itself as an output (weight-only variant): x_h = bf16(u / sqrt(g)) -----
-    if constexpr (!FAST) {
+    {
         if (tn.rot) {                                           // uniform over the CTA
             if (active) {
                 const float2 ig = make_float2(a.inv_sqrt_g, a.inv_sqrt_g);
@@ -428,8 +429,8 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                     reinterpret_cast<uint32_t *>(dst)[0] = w[0];
                 }
             }
-            if constexpr (!FAST && GRID == GRID_UNIFORM) {
-                if (tn.cbf) {
+            if constexpr (GRID == GRID_UNIFORM) {
+                if (tn.cbf) {                                   // uniform over the CTA
                     // a small integer as bfloat16 is the upper half of its binary32 pattern (|c| <= 255: exact)
                     const int L1 = (1 << a.bits) - 1;
                     uint4 *dst = reinterpret_cast<uint4 *>(tn.cbf + row * (long long)cols + (long long)tr * E + g32 * 32);
@@ -930,7 +931,8 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 bool fastw = bits < 8 && trust_factor >= 1.0f;
                 for (int j = 0; j < 2; ++j) {
                     const QuantTensor &t = a.t[j];
-                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && !t.rowsum && !t.rot && !t.cbf)) fastw = false;
+                    const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
+                    if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fastw = false;
                     if (t.rows > 0 && grid_kind == GRID_FP4 && t.op8) fastw = false;
                 }
                 if (grid_kind == GRID_FP4)
@@ -952,7 +954,8 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 bool fast = had_block == 128 && S >= 32 && bits < 8 && trust_factor >= 1.0f;
                 for (int j = 0; j < 2; ++j) {
                     const QuantTensor &t = a.t[j];
-                    if (t.rows > 0 && !(t.codes && t.scales && t.mask && !t.rowsum && !t.rot && !t.cbf)) fast = false;
+                    const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
+                    if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fast = false;
                 }
                 if (grid_kind == GRID_FP4) {
                     // the FP4 codes are the GEMM operand themselves: the specialised path wants codes, scales, mask
