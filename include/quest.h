@@ -59,7 +59,7 @@ typedef enum quest_status {
 enum { QUEST_F32 = 0, QUEST_BF16 = 1 };
 
 /*
- * quest_quantize -- lines 2-3 (or 4-5) of Algorithm 1 for every row of x: the Hadamard
+ * quest_quantize -- the rotation and projection steps of Algorithm 1 for every row of x: the Hadamard
  * rotation of Eq. 2, the RMS normalisation and alpha*(b) clipping of Section 3.1 ("Gaussian
  * Fitting"), rounding onto Eq. 1's b-bit grid, and the trust mask of Section 3.2.
  *
@@ -92,7 +92,7 @@ int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64
                      int bits, int had_block, float trust_factor, uint8_t *mask, void *stream);
 
 /*
- * quest_lowbit_gemm -- line 6 of Algorithm 1 on packed codes: acc[i][j] = sum_k cx[i][k]*cw[j][k]
+ * quest_lowbit_gemm -- the product step of Algorithm 1 on packed codes: acc[i][j] = sum_k cx[i][k]*cw[j][k]
  * in exact int32 (tensor cores, int8 operands), then y[i][j] = sx[i]*sw[j]*acc[i][j]
  * (Section 5: integer matmul with the dequantisation fused into the epilogue).
  *
@@ -148,7 +148,7 @@ int quest_lowbit_gemm_static(const uint8_t *xq, const float *sx, int bits_x,
  *
  *   x [M x K], w [N x K]   device, dense row-major, `dtype`
  *   y [M x N]              device out, dense, `y_dtype`
- *   xq, sx, mx             device out: codes, scales, trust mask of x (Algorithm 1, line 7);
+ *   xq, sx, mx             device out: codes, scales, trust mask of x (the values Algorithm 1 returns);
  *                          xq and sx are required, mx may be NULL
  *   wq, sw, mw             the same for w.  If w_is_cached != 0, w may be NULL and wq/sw are
  *                          INPUTS produced by an earlier call with the same bits and had_block
@@ -231,8 +231,8 @@ int quest_linear_fwd_fp4(const void *x, const void *w, int dtype, int64_t M, int
 
 /*
  * Weight-only variant -- Section 4.5, "Weight-only quantization": the weights are quantized to bits_w
- * bits as in Algorithm 1 (lines 3-4), the activations keep 16 bits.  The paper gives no algorithm of
- * its own for this case; here it is Algorithm 1 with the rounding of line 2 left out:
+ * bits as in Algorithm 1 (its two weight steps), the activations keep 16 bits.  The paper gives no algorithm of
+ * its own for this case; here it is Algorithm 1 with the rounding of the activations left out:
  *   x_h = bf16(HT(x))         every butterfly and the factor 1/sqrt(had_block) in binary32, in the
  *                             quantizer's order, one rounding to bfloat16 (nearest even) at the end
  *   w_q, sw, mw               exactly the outputs of quest_quantize(w, bits_w, had_block, trust_factor)

@@ -3,10 +3,10 @@
 TEST INFRASTRUCTURE ONLY.  Inputs are what the forward pass returns (packed codes, per-row scales,
 trust-mask bitmaps) and the gradient dL/dy:
 
-    dL/dxq_h = dL/dy  wq_h                       (line 2)
-    dL/dx    = IHT( M(x_h; xq_h) * dL/dxq_h )    (line 3)
-    dL/dwq_h = dL/dy^T xq_h                      (line 4)
-    dL/dw    = IHT( M(w_h; wq_h) * dL/dwq_h )    (line 5)
+    dL/dxq_h = dL/dy  wq_h                       (activation-gradient product)
+    dL/dx    = IHT( M(x_h; xq_h) * dL/dxq_h )    (trust mask, inverse transform)
+    dL/dwq_h = dL/dy^T xq_h                      (weight-gradient product)
+    dL/dw    = IHT( M(w_h; wq_h) * dL/dwq_h )    (trust mask, inverse transform)
 
 with xq_h = sx[m] * c_x[m, k] and wq_h = sw[n] * c_w[n, k] the dequantised grid values in the
 orthonormal Hadamard domain (c = 2k - (2^b - 1)), and IHT the inverse of the orthonormal
@@ -65,8 +65,8 @@ def backward(dy: np.ndarray, xq: np.ndarray, sx: np.ndarray, mx: np.ndarray,
     wh = np.asarray(sw, np.float64)[:, None] * grid_values(wq, K, bits)          # wq_h  [N, K]
     rx = np.arange(M) if rows_x is None else np.asarray(rows_x)
     rw = np.arange(N) if rows_w is None else np.asarray(rows_w)
-    d_xh = dy[rx] @ wh                                                            # line 2
-    dx = iht(mask_bits(mx, K)[rx] * d_xh, had_block)                              # line 3
-    d_wh = dy[:, rw].T @ xh                                                       # line 4
-    dw = iht(mask_bits(mw, K)[rw] * d_wh, had_block)                              # line 5
+    d_xh = dy[rx] @ wh                                                            # dL/dxq_h
+    dx = iht(mask_bits(mx, K)[rx] * d_xh, had_block)                              # dL/dx
+    d_wh = dy[:, rw].T @ xh                                                       # dL/dwq_h
+    dw = iht(mask_bits(mw, K)[rw] * d_wh, had_block)                              # dL/dw
     return {"dx": dx, "dw": dw, "d_xh": d_xh, "d_wh": d_wh}

@@ -6,7 +6,7 @@
  * the benchmark's cpu_baseline / reference legs may build, load or call it.  It shares
  * no code, header, table or helper with the CUDA library and never calls it.
  *
- * What it computes, per row x of length d (Algorithm 1, lines 2-6):
+ * What it computes, per row x of length d (Algorithm 1: rotation, projection and product):
  *   1. x_h = HT(x)           Hadamard rotation along the matmul dimension (Eq. 2):
  *                            block-diagonal Sylvester-Hadamard H_g on contiguous blocks
  *                            of g elements, kept UN-normalised (u = H_g * block); the
@@ -19,7 +19,7 @@
  *   4. trust mask            M = [ |x_h - xq_h| <= trust_factor * alpha* * RMS / (2^b-1) ]
  *                            (Section 3.2; the factor s of "The 1-bit Case").
  *   5. y = xq_h wq_h^T       integer contraction of the grid values, then the product of
- *                            the two per-row scales (Algorithm 1, line 6).
+ *                            the two per-row scales (the product step of Algorithm 1).
  *
  * Arithmetic: the paper fixes no precision.  Rounding decisions (codes, masks) are taken
  * in IEEE binary32 with one rounding per operation in a fixed order, stated at each step,
@@ -152,7 +152,7 @@ int qo_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld
         float *tmp = (float *)malloc(sizeof(float) * (size_t)p2);
 #pragma omp for schedule(static)
         for (int64_t r = 0; r < rows; ++r) {
-            /* line 2 / 4 of Algorithm 1: rotate */
+            /* Algorithm 1, rotation step (x_h = HT(x), w_h = HT(w)) */
             if (dtype == 0) {
                 const float *xr = (const float *)x + r * ld;
                 for (int64_t e = 0; e < cols; ++e) u[e] = xr[e];
@@ -174,7 +174,7 @@ int qo_quantize(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld
             if (cr) memset(cr, 0, (size_t)code_row_bytes);
             if (mr) memset(mr, 0, (size_t)mask_row_bytes);
             for (int64_t e = 0; e < cols; ++e) {
-                /* line 3 / 5: clip to [-alpha*, alpha*] RMS and round to the nearest of the
+                /* Algorithm 1, projection step: clip to [-alpha*, alpha*] RMS and round to the nearest of the
                  * 2^b grid points; on the level axis the grid points are the integers
                  * 0..L1.  READING: ties go to the even level (rintf, default mode). */
                 const float t = fmaf(u[e], inv, c0);
@@ -214,7 +214,7 @@ int qo_unpack_grid_values(const uint8_t *codes, int64_t rows, int64_t cols, int 
     return QO_OK;
 }
 
-/* Algorithm 1, line 6, integer part: acc[i][j] = sum_k cx[i][k] * cw[j][k], exact.
+/* Algorithm 1, product step, integer part: acc[i][j] = sum_k cx[i][k] * cw[j][k], exact.
  * Accumulated in 64 bits and checked to fit 32. */
 int qo_gemm_acc(const uint8_t *xq, int bits_x, const uint8_t *wq, int bits_w,
                 int64_t M, int64_t N, int64_t K, int32_t *acc) {
@@ -242,7 +242,7 @@ int qo_gemm_acc(const uint8_t *xq, int bits_x, const uint8_t *wq, int bits_w,
     return status;
 }
 
-/* Algorithm 1, line 6, scale part: y[i][j] = sx[i] * sw[j] * acc[i][j] in binary64. */
+/* Algorithm 1, product step, scale part: y[i][j] = sx[i] * sw[j] * acc[i][j] in binary64. */
 int qo_dequant(const int32_t *acc, const float *sx, const float *sw, int64_t M, int64_t N, double *y) {
     if (!acc || !sx || !sw || !y) return QO_BAD_ARG;
     for (int64_t i = 0; i < M; ++i)

@@ -3,8 +3,8 @@
 TEST INFRASTRUCTURE ONLY.  The paper trains models whose weights are quantized to 1-4 bits while
 the activations keep 16 bits, and gives no separate algorithm for it.
 
-READING: Algorithm 1 with the rounding of the activations (line 2) left out.  The weights take
-lines 3-4 unchanged (rotation, RMS scale, rounding to the b-bit grid: ``quest_oracle.quantize``).
+READING: Algorithm 1 with the rounding of the activations left out.  The weights take their two
+steps unchanged (rotation, then RMS scale and rounding to the b-bit grid: ``quest_oracle.quantize``).
 The activations are rotated by the same orthonormal block Hadamard transform and stored as
 bfloat16, the 16-bit activation type of the paper's runs:
 

@@ -269,7 +269,7 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
     }
     if (dx) {
         Stage gemm_stage(QUEST_STAGE_GEMM, st);
-        // line 2 and the mask of line 3: d1[m][k] = M_x[m][k] * sum_n dy[m][n] wq_h[n][k]
+        // activation gradient of Algorithm 2 with its trust mask: d1[m][k] = M_x[m][k] * sum_n dy[m][n] wq_h[n][k]
         // (blocks of 128: the inverse transform is fused into the contraction's epilogue)
         if (had_block == 128 && M > 128 && K > 128) {
             if ((s = launch_gemm_bf16_masked(dy, ws.wh, M, K, N, mx, dx, out_dtype, true, 1, st))) return s;
@@ -280,7 +280,7 @@ extern "C" int quest_linear_bwd(const void *dy, int64_t M, int64_t N, int64_t K,
     }
     if (dw) {
         Stage gemm_stage(QUEST_STAGE_GEMM, st);
-        // line 4 and the mask of line 5: d2[n][k] = M_w[n][k] * sum_m dy[m][n] xq_h[m][k]
+        // weight gradient of Algorithm 2 with its trust mask: d2[n][k] = M_w[n][k] * sum_m dy[m][n] xq_h[m][k]
         if (had_block == 128 && N > 128 && K > 128) {
             if ((s = launch_gemm_bf16_masked(dy, ws.xh, N, K, M, mw, dw, out_dtype, true, 2, st))) return s;
         } else {

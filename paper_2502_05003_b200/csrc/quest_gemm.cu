@@ -1,4 +1,4 @@
-// Low-bit GEMM of the QuEST forward pass (Algorithm 1, line 6; Section 5, stage 3) for sm_100a.
+// Low-bit GEMM of the QuEST forward pass (the product step of Algorithm 1; Section 5, stage 3) for sm_100a.
 //
 //   acc[i][j] = sum_k cx[i][k] * cw[j][k]   exact int32, 5th-generation tensor cores
 //   y[i][j]   = sx[i] * sw[j] * acc[i][j]   fused into the epilogue, bf16 or fp32 out
@@ -584,7 +584,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 else mbar_arrive(smem_u32(&tempty_bar[buf]));
             }
             if constexpr (IHT128) {
-                // lines 3 / 5 of Algorithm 2 on this thread's block of 128: mask, then the inverse
+                // trust mask and inverse transform of Algorithm 2 on this thread's block of 128: mask, then the inverse
                 // orthonormal Hadamard transform in registers (descending stride, packed binary32)
                 if (n0 + cbase < p.N) {
                     uint4 mb = make_uint4(0u, 0u, 0u, 0u);
@@ -1024,7 +1024,7 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
 #undef QUEST_GEMM
 }
 
-// Backward-pass contraction (Algorithm 2, lines 2 and 4): out[i][j] = mask[i][j] * sum_k A(i, k) B(j, k) with
+// Backward-pass contraction (the two products of Algorithm 2): out[i][j] = mask[i][j] * sum_k A(i, k) B(j, k) with
 // bfloat16 operands and binary32 output [I x J].  `opl` says how the operands lie in memory:
 //   0: a [I x Kc], b [J x Kc], the contraction index contiguous (K-major);
 //   1: a [I x Kc] K-major, b [Kc x J] (memory rows run along the contraction: MN-major);

@@ -1,6 +1,6 @@
 // Fused QuEST forward quantizer for sm_100a: Hadamard rotation (Eq. 2) -> RMS normalisation ->
 // alpha*(b) clip -> round onto Eq. 1's grid -> packed codes, per-row scale, trust mask
-// (Section 3.1 and 3.2; lines 2-5 of Algorithm 1).
+// (Section 3.1 and 3.2; the rotation and projection steps of Algorithm 1).
 //
 // Every rounding decision is taken in binary32 with one IEEE rounding per operation, in this
 // order: butterflies (a,b) -> (a+b, a-b) with DESCENDING stride g/2 .. 1; squares rounded, then

@@ -1,4 +1,4 @@
-"""Pins for Algorithm 1 line 6 in the oracle: the integer contraction and the scale product."""
+"""Pins for the product step of Algorithm 1 in the oracle: the integer contraction and the scale product."""
 import numpy as np
 import pytest
 
