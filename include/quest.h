@@ -178,7 +178,7 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
  *
  * with the trust estimator of Section 3.2 applied in the Hadamard domain and IHT the inverse of
  * the orthonormal block Hadamard transform.  The two products run on the tensor cores with
- * bfloat16 operands and binary32 accumulation ("standard 16-bit precision", Section 3.3): dL/dy as
+ * bfloat16 operands and binary32 accumulation (Section 3.3 keeps the backward products in 16 bits): dL/dy as
  * given, the quantized operand dequantised to bfloat16 (scale * grid value, one rounding per element).
  *
  *   dy                 device, [M x N] bfloat16, dense, 16-byte aligned
