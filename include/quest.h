@@ -1,11 +1,14 @@
 /*
- * quest.h -- C ABI of the B200 (sm_100a) QuEST quantized-linear forward library.
+ * quest.h -- C ABI of the B200 (sm_100a) QuEST quantized-linear library.
  *
  * The library implements the forward pass of one QuEST linear layer (Algorithm 1 of
  * "QuEST: Stable Training of LLMs with 1-Bit Weights and Activations", arXiv 2502.05003):
  *
  *     x_h = HT(x);  xq_h = proj_{alpha*}(x_h);  w_h = HT(w);  wq_h = proj_{alpha*}(w_h);
  *     y   = xq_h wq_h^T;   return y, xq_h, wq_h, M(x_h; xq_h), M(w_h; wq_h)
+ *
+ * and, further down, its backward pass (Algorithm 2), the FP4 grid of Section 4.4 and the
+ * weight-only variant of Section 4.5.
  *
  * General rules for every entry point
  *   - Pointers named in "device" are CUDA device pointers owned by the caller; the library
@@ -93,8 +96,10 @@ int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64
 
 /*
  * quest_lowbit_gemm -- the product step of Algorithm 1 on packed codes: acc[i][j] = sum_k cx[i][k]*cw[j][k]
- * in exact int32 (tensor cores, int8 operands), then y[i][j] = sx[i]*sw[j]*acc[i][j]
- * (Section 5: integer matmul with the dequantisation fused into the epilogue).
+ * exactly, reported as int32 (tensor cores: int8 operands, or E2M1 operands on the FP4 path when both
+ * widths are at most 2, whose grid values +-1 and +-3 are E2M1 numbers), then
+ * y[i][j] = sx[i]*sw[j]*acc[i][j] (Section 5: integer matmul with the dequantisation fused into the
+ * epilogue).
  *
  *   xq, sx, bits_x   device: codes [M x K] and scales [M] of the activations
  *   wq, sw, bits_w   device: codes [N x K] and scales [N] of the weights (both operands K-major)
@@ -103,7 +108,7 @@ int quest_trust_mask(const void *x, int dtype, int64_t rows, int64_t cols, int64
  *                    may be NULL if only acc is wanted
  *   acc              device out, dense [M x N] int32 raw accumulators; may be NULL
  *   workspace        device scratch of at least quest_workspace_bytes(M, N, K, bits_x, bits_w)
- *                    bytes, 256-byte aligned; holds the int8 operands the tensor cores read.
+ *                    bytes, 256-byte aligned; holds the operands the tensor cores read.
  *                    Its contents are undefined afterwards; two calls that overlap on the GPU
  *                    must not share it.
  */
