@@ -254,6 +254,20 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 
 constexpr int MAX_STAGES = 6;
 
+// Tile order: m fastest inside bands of RASTER_M row tiles, bands one after another.  Concurrent CTAs
+// then share one or two column tiles of B while the rows of A a band touches (RASTER_M x TILE_M x K
+// bytes) stay in L2 for all of the band's column tiles; with a single band (up to RASTER_M row tiles)
+// this is plain column-major order.
+constexpr int RASTER_M = 16;
+__device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int &tm, int &tn) {
+    const int band_tiles = RASTER_M * num_n;
+    const int band = tile / band_tiles;
+    const int t = tile - band * band_tiles;
+    const int rows_here = min(RASTER_M, num_m - band * RASTER_M);
+    tn = t / rows_here;
+    tm = band * RASTER_M + (t - tn * rows_here);
+}
+
 // 32 columns of this warp's 32 TMEM lanes, issued without waiting: the registers are valid only
 // after tmem_wait_ld() and pin() (an empty volatile asm that makes every later use depend on a
 // statement ordered after the wait).
@@ -402,8 +416,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
-                const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;          // this CTA's rows of A
-                const int n0 = (tile / num_m) * BN + (int)rank * L::B_ROWS;      // this CTA's rows of B
+                int tm, tn;
+                tile_coords(tile, num_m, num_n, tm, tn);
+                const int m0 = tm * TILE_M + (int)rank * BM;                     // this CTA's rows of A
+                const int n0 = tn * BN + (int)rank * L::B_ROWS;                  // this CTA's rows of B
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, p.status, ST_PRODUCER);
                     if (!ok) break;
@@ -527,8 +543,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint8_t *slab_base = smem + L::STG_OFFSET + (warp - 2) * (L::SLABS * 4096);
         int slab_count = 0;                            // slabs this warp has handed to TMA
         for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
-            const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
-            const int n0 = (tile / num_m) * BN;
+            int tm, tn;
+            tile_coords(tile, num_m, num_n, tm, tn);
+            const int m0 = tm * TILE_M + (int)rank * BM;
+            const int n0 = tn * BN;
             const int buf = NBUF == 2 ? (t & 1) : 0;
             const uint32_t bphase = (uint32_t)(NBUF == 2 ? (t >> 1) : t) & 1u;
             // stage this tile's column scales (and column corrections) in shared memory; the
