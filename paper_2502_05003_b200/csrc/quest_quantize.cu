@@ -878,8 +878,10 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
         int S;
         if (T < 32) { S = 1; while (S < T) S <<= 1; } else { S = (T + 31) / 32 * 32; }
         // rows per CTA: 128-thread CTAs for the 32-per-thread streaming kernel (eight per SM) measured 4-10 % faster
-        // than 256-thread ones: finer work units at the tail and fewer warps behind each CTA-wide barrier
-        const int R = (stream32 && S <= 128) ? 128 / S : (S >= 256 ? 1 : 256 / S);
+        // than 256-thread ones (finer work units at the tail, fewer warps behind each CTA-wide barrier), and
+        // 14-38 % faster for the direct-load kernel (binary32 rows, blocks below 64)
+        const bool direct = dtype != QUEST_BF16 || had_block < 64;
+        const int R = ((stream32 || direct) && S <= 128) ? 128 / S : (S >= 256 ? 1 : 256 / S);
         const int threads = R * S;
         const int warps = (threads + 31) / 32;
         const size_t smem = had_block >= 64 * E ? sizeof(float) * E * (size_t)threads : sizeof(float) * (size_t)warps;
