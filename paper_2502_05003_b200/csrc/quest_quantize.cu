@@ -798,6 +798,64 @@ static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaS
 #undef QUEST_LAUNCH
 }
 
+// The specialised case (bfloat16 rows, had_block = 128, 32 elements per thread) with direct loads and
+// one CTA per row group: at sizes whose whole input is a few waves of CTAs the hardware's own CTA
+// scheduling balances better than the persistent loop of the streaming kernel and there is no
+// staging to set up.  Stride 64 pairs this thread with lane ^ 2 (shuffles); the rest is the common tail.
+template <int CB, int GRID = GRID_UNIFORM>
+__global__ void __launch_bounds__(256, 4)
+quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
+    extern __shared__ float xsm[];                 // [warps] partial sums
+    pdl_launch_dependents();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
+    const QuantTensor &tn = a.t[which];
+    const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
+    const int r_local = tid / a.S;
+    const int tr = tid - r_local * a.S;
+    const long long row = (long long)blk * a.R + r_local;
+    const bool active = row < tn.rows && tr < (a.cols >> 5);   // slots past the row end hold zeros
+    float2 v[16];
+    if (active) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(tn.x) + row * tn.ld + (long long)tr * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint4 w = __ldg(src + q);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                v[q * 4 + j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = make_float2(0.0f, 0.0f);
+    }
+    {
+        const float sg = (lane & 2) ? -1.0f : 1.0f;
+        const float2 sgn = make_float2(sg, sg);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            float2 p;
+            p.x = __shfl_xor_sync(0xffffffffu, v[i].x, 2);
+            p.y = __shfl_xor_sync(0xffffffffu, v[i].y, 2);
+            v[i] = __ffma2_rn(v[i], sgn, p);
+        }
+    }
+    rotate_project_store<CB, 32, true, true, GRID>(v, a, tn, active, row, tr, r_local, xsm, 32);
+}
+
+template <int GRID>
+static cudaError_t launch_direct128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
+    if (GRID == GRID_FP4) return launch_pdl(quantize_direct128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
+    switch (cb) {
+        case 1: return launch_pdl(quantize_direct128_kernel<1, GRID>, grid, dim3(threads), smem, st, 1, a);
+        case 2: return launch_pdl(quantize_direct128_kernel<2, GRID>, grid, dim3(threads), smem, st, 1, a);
+        case 4: return launch_pdl(quantize_direct128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
+        default: return launch_pdl(quantize_direct128_kernel<8, GRID>, grid, dim3(threads), smem, st, 1, a);
+    }
+}
+
 template <bool BF16, int E>
 static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
@@ -870,18 +928,17 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
     if (grid_kind == GRID_FP4 && cols % 32 != 0) return QUEST_ERR_SHAPE;
     const int cb = container_bits(bits);
     if (cols % 32 == 0) {
-        // streaming kernel with 32 elements per thread (64 registers, twice the resident warps) measured
-        // faster than 64 per thread for rows up to 4096 elements; wider rows keep 64 per thread
-        const bool stream32 = dtype == QUEST_BF16 && had_block >= 64 && cols <= 4096;
-        const int E = (cols % 64 == 0 && !stream32) ? 64 : 32;
+        // 32 elements per thread (64 registers, twice the resident warps) for bfloat16 rows up to 8192 elements;
+        // wider rows keep 64 per thread
+        const bool e32 = dtype == QUEST_BF16 && had_block >= 64 && cols <= 8192;
+        const int E = (cols % 64 == 0 && !e32) ? 64 : 32;
         const int T = (int)(cols / E);
         int S;
         if (T < 32) { S = 1; while (S < T) S <<= 1; } else { S = (T + 31) / 32 * 32; }
-        // rows per CTA: 128-thread CTAs for the 32-per-thread streaming kernel (eight per SM) measured 4-10 % faster
-        // than 256-thread ones (finer work units at the tail, fewer warps behind each CTA-wide barrier), and
-        // 14-38 % faster for the direct-load kernel (binary32 rows, blocks below 64)
-        const bool direct = dtype != QUEST_BF16 || had_block < 64;
-        const int R = ((stream32 || direct) && S <= 128) ? 128 / S : (S >= 256 ? 1 : 256 / S);
+        // rows per CTA: CTAs of 128 threads wherever a row fits (finer work units, fewer warps behind each
+        // CTA-wide barrier) except for the persistent 64-per-thread streaming kernel
+        const bool streaming = E == 64 && dtype == QUEST_BF16 && had_block >= 64;
+        const int R = (!streaming && S <= 128) ? 128 / S : (S >= 256 ? 1 : 256 / S);
         const int threads = R * S;
         const int warps = (threads + 31) / 32;
         const size_t smem = had_block >= 64 * E ? sizeof(float) * E * (size_t)threads : sizeof(float) * (size_t)warps;
@@ -907,77 +964,58 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             a.inv_sqrt_g = 1.0f / sqrtf((float)had_block);
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
-            const bool streaming = (E == 64 || stream32) && dtype == QUEST_BF16 && had_block >= 64;
-            if (grid_kind == GRID_FP4 && !streaming) {
+            // the specialised tail: codes, scales and masks requested (or the rotation alone), trust_factor >= 1,
+            // below 8 bits; the FP4 grid has no separate GEMM operand
+            bool fast_tail = bits < 8 && trust_factor >= 1.0f && S >= 32;
+            for (int j = 0; j < 2; ++j) {
+                const QuantTensor &t = a.t[j];
+                const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
+                if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fast_tail = false;
+                if (t.rows > 0 && grid_kind == GRID_FP4 && (t.op8 || t.rot || t.cbf)) fast_tail = false;
+            }
+            int dev = 0, sms = 148;
+            cudaGetDevice(&dev);
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            const int total = nb[0] + nb[1];
+            if (e32 && S == T && S <= 256 && (had_block == 1024 || had_block == 2048 || had_block == 4096)) {
+                // wide rotation blocks: layout-change kernel (persistent, double-buffered raw rows)
+                const int exchange = (int)((sizeof(float) * (size_t)warps + 15) / 16 * 16);
+                const size_t smem2 = (size_t)exchange + (size_t)R * (cols + cols / 8) * 4 + 2 * (size_t)R * cols * 2;
+                int per_sm = (int)((220 * 1024) / (smem2 + 1024));
+                const int by_threads = 1024 / threads;
+                if (per_sm > by_threads) per_sm = by_threads;
+                if (per_sm < 1) per_sm = 1;
+                const int g = total < sms * per_sm ? total : sms * per_sm;
+                if (grid_kind == GRID_FP4)
+                    e = fast_tail ? launch_wide<GRID_FP4, true>(cb, g, threads, smem2, st, a, total, exchange)
+                                  : launch_wide<GRID_FP4, false>(cb, g, threads, smem2, st, a, total, exchange);
+                else
+                    e = fast_tail ? launch_wide<GRID_UNIFORM, true>(cb, g, threads, smem2, st, a, total, exchange)
+                                  : launch_wide<GRID_UNIFORM, false>(cb, g, threads, smem2, st, a, total, exchange);
+            } else if (e32 && had_block == 128 && fast_tail && threads <= 256) {
+                // the common case: direct loads, one CTA per row group
+                e = grid_kind == GRID_FP4 ? launch_direct128<GRID_FP4>(cb, grid, threads, smem, st, a)
+                                          : launch_direct128<GRID_UNIFORM>(cb, grid, threads, smem, st, a);
+            } else if (streaming) {
+                // rows wider than 8192: persistent streaming kernel, 64 elements per thread, as many CTAs as fit
+                const int exchange = (int)((smem + 15) / 16 * 16);
+                const size_t smem2 = (size_t)exchange + 2 * (size_t)threads * (2 * E + 16);
+                const int per_sm = smem2 > 100 * 1024 ? 1 : 2;
+                const int g = total < sms * per_sm ? total : sms * per_sm;
+                const bool fast = fast_tail && had_block == 128;
+                if (grid_kind == GRID_FP4)
+                    e = fast ? launch_stream_fp4<64, true>(g, threads, smem2, st, a, total, exchange)
+                             : launch_stream_fp4<64, false>(g, threads, smem2, st, a, total, exchange);
+                else
+                    e = fast ? launch_stream<64, true>(cb, g, threads, smem2, st, a, total, exchange)
+                             : launch_stream<64, false>(cb, g, threads, smem2, st, a, total, exchange);
+            } else if (grid_kind == GRID_FP4) {
                 if (E == 64)
                     e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 64>(grid, threads, smem, st, a)
                                             : launch_rows_fp4<false, 64>(grid, threads, smem, st, a);
                 else
                     e = dtype == QUEST_BF16 ? launch_rows_fp4<true, 32>(grid, threads, smem, st, a)
                                             : launch_rows_fp4<false, 32>(grid, threads, smem, st, a);
-            } else if (streaming && E == 32 && S == T && S <= 256 &&
-                       (had_block == 1024 || had_block == 2048 || had_block == 4096)) {
-                // wide rotation blocks: layout-change kernel (persistent, double-buffered raw rows)
-                const int exchange = (int)((sizeof(float) * (size_t)warps + 15) / 16 * 16);
-                const size_t smem2 = (size_t)exchange + (size_t)R * (cols + cols / 8) * 4 + 2 * (size_t)R * cols * 2;
-                int dev = 0, sms = 148;
-                cudaGetDevice(&dev);
-                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-                int per_sm = (int)((220 * 1024) / (smem2 + 1024));
-                const int by_threads = 1024 / threads;
-                if (per_sm > by_threads) per_sm = by_threads;
-                if (per_sm < 1) per_sm = 1;
-                const int total = nb[0] + nb[1];
-                const int g = total < sms * per_sm ? total : sms * per_sm;
-                // the specialised tail (codes, scales and masks requested, trust_factor >= 1, below 8 bits)
-                bool fastw = bits < 8 && trust_factor >= 1.0f;
-                for (int j = 0; j < 2; ++j) {
-                    const QuantTensor &t = a.t[j];
-                    const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
-                    if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fastw = false;
-                    if (t.rows > 0 && grid_kind == GRID_FP4 && t.op8) fastw = false;
-                }
-                if (grid_kind == GRID_FP4)
-                    e = fastw ? launch_wide<GRID_FP4, true>(cb, g, threads, smem2, st, a, total, exchange)
-                              : launch_wide<GRID_FP4, false>(cb, g, threads, smem2, st, a, total, exchange);
-                else
-                    e = fastw ? launch_wide<GRID_UNIFORM, true>(cb, g, threads, smem2, st, a, total, exchange)
-                              : launch_wide<GRID_UNIFORM, false>(cb, g, threads, smem2, st, a, total, exchange);
-            } else if (streaming) {
-                // persistent streaming kernel: as many CTAs as fit on the device, each looping over groups
-                const int exchange = (int)((smem + 15) / 16 * 16);
-                const size_t smem2 = (size_t)exchange + 2 * (size_t)threads * (2 * E + 16);
-                int dev = 0, sms = 148;
-                cudaGetDevice(&dev);
-                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-                const int per_sm = smem2 > 100 * 1024 ? 1 : (E == 64 ? 2 : (threads <= 128 ? 8 : 4));
-                const int total = nb[0] + nb[1];
-                const int g = total < sms * per_sm ? total : sms * per_sm;
-                bool fast = had_block == 128 && S >= 32 && bits < 8 && trust_factor >= 1.0f;
-                for (int j = 0; j < 2; ++j) {
-                    const QuantTensor &t = a.t[j];
-                    const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
-                    if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fast = false;
-                }
-                if (grid_kind == GRID_FP4) {
-                    // the FP4 codes are the GEMM operand themselves: the specialised path wants codes, scales, mask
-                    bool fast4 = had_block == 128 && S >= 32 && trust_factor >= 1.0f;
-                    for (int j = 0; j < 2; ++j) {
-                        const QuantTensor &t = a.t[j];
-                        if (t.rows > 0 && !(t.codes && t.scales && t.mask && !t.op8 && !t.rowsum && !t.rot && !t.cbf)) fast4 = false;
-                    }
-                    if (fast4)
-                        e = E == 64 ? launch_stream_fp4<64, true>(g, threads, smem2, st, a, total, exchange)
-                                    : launch_stream_fp4<32, true>(g, threads, smem2, st, a, total, exchange);
-                    else
-                        e = E == 64 ? launch_stream_fp4<64, false>(g, threads, smem2, st, a, total, exchange)
-                                    : launch_stream_fp4<32, false>(g, threads, smem2, st, a, total, exchange);
-                } else if (fast)
-                    e = E == 64 ? launch_stream<64, true>(cb, g, threads, smem2, st, a, total, exchange)
-                                : launch_stream<32, true>(cb, g, threads, smem2, st, a, total, exchange);
-                else
-                    e = E == 64 ? launch_stream<64, false>(cb, g, threads, smem2, st, a, total, exchange)
-                                : launch_stream<32, false>(cb, g, threads, smem2, st, a, total, exchange);
             } else if (E == 64)
                 e = dtype == QUEST_BF16 ? launch_rows<true, 64>(cb, grid, threads, smem, st, a)
                                         : launch_rows<false, 64>(cb, grid, threads, smem, st, a);
