@@ -43,8 +43,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this command's
 # kernels (None when no capture of the current kernel exists).
 GEMM_DRAM_TRAFFIC_BYTES = 12652032          # low-bit GEMM, 4096 x 2048 x 2048
-QUANT_DRAM_TRAFFIC_BYTES = 25189376         # quantizer, x and w in one launch
-QUANT_INSTR_PER_ELEMENT = 24.7              # thread instructions per element, same capture
+QUANT_DRAM_TRAFFIC_BYTES = 25191168         # quantizer, x and w in one launch
+QUANT_INSTR_PER_ELEMENT = 23.3              # thread instructions per element, same capture
 
 
 def load_peaks():
