@@ -636,7 +636,7 @@ quantize_stream_kernel(const __grid_constant__ QuantArgs a, int total_groups, in
 // Wide rotation blocks (had_block = 1024, 2048 or 4096, bfloat16 rows): the five largest strides are
 // made thread-local by a change of data layout instead of five rounds of warp shuffles.  A block of
 // g = 32 G elements belongs to G threads.  Phase A: thread p of the block takes the 32 elements
-// p + G j (j = 0..31) from the raw row in shared memory, so the strides g/2 .. g/32 pair elements
+// p + G j (j = 0..31) of the row straight from global memory, so the strides g/2 .. g/32 pair elements
 // it already holds (one in-register 32-point butterfly, largest stride first).  The result goes
 // back to shared memory in row order (binary32, 16 bytes of padding per 32 elements).  Phase B:
 // every thread reads its 32 contiguous elements; the one or two strides left between g/64 and 32
@@ -664,7 +664,7 @@ __device__ __forceinline__ void butterfly32_in_registers(float2 (&v)[16]) {
 
 template <int CB, bool FAST, int GRID = GRID_UNIFORM>
 __global__ void __launch_bounds__(256, 3)
-quantize_wide_kernel(const __grid_constant__ QuantArgs a, int total_groups, int exchange_bytes) {
+quantize_wide_kernel(const __grid_constant__ QuantArgs a, int exchange_bytes) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     pdl_launch_dependents();
     pdl_wait();
@@ -674,54 +674,30 @@ quantize_wide_kernel(const __grid_constant__ QuantArgs a, int total_groups, int 
     float *xsm = reinterpret_cast<float *>(smem_raw);
     float *tbuf = reinterpret_cast<float *>(smem_raw + exchange_bytes);
     const int trow_words = cols + (cols >> 3);                 // 36 words per 32 elements
-    uint8_t *raw = reinterpret_cast<uint8_t *>(tbuf + (size_t)R * trow_words);
     const int tid = threadIdx.x;
     const int r_local = tid / S;
     const int tr = tid - r_local * S;
     const int p = tr & (G - 1);
     const int blk_base = (tr >> gshift) * a.had_block;         // first element of this thread's block
-
-    auto locate = [&](int grp, int &which, long long &row) {
-        which = grp >= a.blocks0 ? 1 : 0;
-        row = (long long)(which ? grp - a.blocks0 : grp) * R + r_local;
-    };
-    auto prefetch = [&](int grp, int buf) {
-        if (grp < total_groups) {
-            int which;
-            long long row;
-            locate(grp, which, row);
-            const QuantTensor &tn = a.t[which];
-            const bool live = row < tn.rows;
-            const uint8_t *src = live ? reinterpret_cast<const uint8_t *>(tn.x) + (row * tn.ld + (long long)tr * 32) * 2
-                                      : reinterpret_cast<const uint8_t *>(tn.x);
-            const uint32_t nbytes = live ? 16u : 0u, step = live ? 16u : 0u;
-            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(raw + ((size_t)(buf * R + r_local) * cols + (size_t)tr * 32) * 2);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + q * 16), "l"(src + q * step), "r"(nbytes)
-                             : "memory");
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-
-    int buf = 0;
-    prefetch((int)blockIdx.x, 0);
-    for (int grp = (int)blockIdx.x; grp < total_groups; grp += (int)gridDim.x, buf ^= 1) {
-        prefetch(grp + (int)gridDim.x, buf ^ 1);
-        asm volatile("cp.async.wait_group 1;" ::: "memory");
-        __syncthreads();                                       // the whole row has landed; last round's readers are done
-        int which;
-        long long row;
-        locate(grp, which, row);
+    {
+        const int grp = (int)blockIdx.x;                       // one CTA per group of R rows
+        const int which = grp >= a.blocks0 ? 1 : 0;
+        const long long row = (long long)(which ? grp - a.blocks0 : grp) * R + r_local;
         const QuantTensor &tn = a.t[which];
         const bool active = row < tn.rows;
         float2 v[16];
         {   // phase A: elements p + G j of this thread's block, then strides g/2 .. g/32 in registers
-            const uint16_t *rrow = reinterpret_cast<const uint16_t *>(raw + (size_t)(buf * R + r_local) * cols * 2) + blk_base + p;
+            // (two-byte loads: a warp reads 64 contiguous bytes per instruction, every byte once)
+            if (active) {
+                const uint16_t *rrow = reinterpret_cast<const uint16_t *>(tn.x) + row * tn.ld + blk_base + p;
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-                v[j] = make_float2(__uint_as_float((uint32_t)rrow[(2 * j) << gshift] << 16),
-                                   __uint_as_float((uint32_t)rrow[(2 * j + 1) << gshift] << 16));
+                for (int j = 0; j < 16; ++j)
+                    v[j] = make_float2(__uint_as_float((uint32_t)__ldg(rrow + ((2 * j) << gshift)) << 16),
+                                       __uint_as_float((uint32_t)__ldg(rrow + ((2 * j + 1) << gshift)) << 16));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = make_float2(0.0f, 0.0f);
+            }
             butterfly32_in_registers(v);
             float *trow = tbuf + (size_t)r_local * trow_words;
 #pragma unroll
@@ -774,19 +750,18 @@ quantize_wide_kernel(const __grid_constant__ QuantArgs a, int total_groups, int 
         }
         rotate_project_store<CB, 32, true, FAST, GRID, true>(v, a, tn, active, row, tr, r_local, xsm, 16);
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 template <int GRID, bool FAST>
 static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
-                               int total_groups, int exchange_bytes) {
+                               int exchange_bytes) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
         cudaError_t e_ = cudaFuncSetAttribute(quantize_wide_kernel<CBV, FAST, GRID>,                        \
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);     \
         if (e_ != cudaSuccess) return e_;                                                                   \
         return launch_pdl(quantize_wide_kernel<CBV, FAST, GRID>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
-                          total_groups, exchange_bytes);                                                    \
+                          exchange_bytes);                                                                  \
     } while (0)
     if (GRID == GRID_FP4) QUEST_LAUNCH(4);
     switch (cb) {
@@ -978,20 +953,16 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
             const int total = nb[0] + nb[1];
             if (e32 && S == T && S <= 256 && (had_block == 1024 || had_block == 2048 || had_block == 4096)) {
-                // wide rotation blocks: layout-change kernel (persistent, double-buffered raw rows)
+                // wide rotation blocks: layout-change kernel, one CTA per row group
                 const int exchange = (int)((sizeof(float) * (size_t)warps + 15) / 16 * 16);
-                const size_t smem2 = (size_t)exchange + (size_t)R * (cols + cols / 8) * 4 + 2 * (size_t)R * cols * 2;
-                int per_sm = (int)((220 * 1024) / (smem2 + 1024));
-                const int by_threads = 1024 / threads;
-                if (per_sm > by_threads) per_sm = by_threads;
-                if (per_sm < 1) per_sm = 1;
-                const int g = total < sms * per_sm ? total : sms * per_sm;
+                const size_t smem2 = (size_t)exchange + (size_t)R * (cols + cols / 8) * 4;
+                const int g = total;
                 if (grid_kind == GRID_FP4)
-                    e = fast_tail ? launch_wide<GRID_FP4, true>(cb, g, threads, smem2, st, a, total, exchange)
-                                  : launch_wide<GRID_FP4, false>(cb, g, threads, smem2, st, a, total, exchange);
+                    e = fast_tail ? launch_wide<GRID_FP4, true>(cb, g, threads, smem2, st, a, exchange)
+                                  : launch_wide<GRID_FP4, false>(cb, g, threads, smem2, st, a, exchange);
                 else
-                    e = fast_tail ? launch_wide<GRID_UNIFORM, true>(cb, g, threads, smem2, st, a, total, exchange)
-                                  : launch_wide<GRID_UNIFORM, false>(cb, g, threads, smem2, st, a, total, exchange);
+                    e = fast_tail ? launch_wide<GRID_UNIFORM, true>(cb, g, threads, smem2, st, a, exchange)
+                                  : launch_wide<GRID_UNIFORM, false>(cb, g, threads, smem2, st, a, exchange);
             } else if (e32 && had_block == 128 && fast_tail && threads <= 256) {
                 // the common case: direct loads, one CTA per row group
                 e = grid_kind == GRID_FP4 ? launch_direct128<GRID_FP4>(cb, grid, threads, smem, st, a)
