@@ -268,8 +268,9 @@ int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
     {
         StageScope scope(QUEST_STAGE_UNPACK, st);
         const bool e4 = e2m1_operands(bits_x, bits_w);
-        if ((s = launch_unpack(xq, bits_x, M, K, ws.a8, need_rs_a ? ws.rs_a : nullptr, st, e4))) return s;
-        if ((s = launch_unpack(wq, bits_w, N, K, ws.b8, need_rs_b ? ws.rs_b : nullptr, st, e4))) return s;
+        if ((s = launch_unpack_pair(xq, bits_x, M, ws.a8, need_rs_a ? ws.rs_a : nullptr, wq, bits_w, N, ws.b8,
+                                    need_rs_b ? ws.rs_b : nullptr, K, e4, st)))
+            return s;
     }
     StageScope scope(QUEST_STAGE_GEMM, st);
     return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits_x, bits_w, sx, sw, M, N, K, y, y_dtype, ldy_elems, acc,

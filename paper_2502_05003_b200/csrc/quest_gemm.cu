@@ -849,6 +849,47 @@ __global__ void unpack_codes_e2m1_kernel(const uint8_t *__restrict__ codes, long
     }
 }
 
+// Both operands of a contraction in one launch (each with its own width): thread g converts 32
+// consecutive elements of x when g < groups_x, else of w.
+template <int CB>
+__device__ __forceinline__ void unpack_group(const uint8_t *codes, int bits, long long g, uint8_t *out, bool e2m1) {
+    uint32_t w[CB];
+#pragma unroll
+    for (int q = 0; q < CB; ++q) w[q] = __ldg(reinterpret_cast<const uint32_t *>(codes) + g * CB + q);
+    if constexpr (CB <= 2) {
+        if (e2m1) {
+            uint32_t o[4];
+            e2m1_operand_from_code_words<CB>(w, o);
+            *reinterpret_cast<uint4 *>(out + g * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+            return;
+        }
+    }
+    uint32_t o[8];
+    operand_from_code_words<CB>(w, bits, o);
+    uint4 *dst = reinterpret_cast<uint4 *>(out + g * 32);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+__global__ void __launch_bounds__(128)
+unpack_pair_kernel(const uint8_t *__restrict__ codes_x, int bits_x, long long groups_x, uint8_t *__restrict__ out_x,
+                   const uint8_t *__restrict__ codes_w, int bits_w, long long groups_w, uint8_t *__restrict__ out_w, int e2m1) {
+    pdl_launch_dependents();
+    pdl_wait();
+    long long g = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (g >= groups_x + groups_w) return;
+    const bool second = g >= groups_x;
+    if (second) g -= groups_x;
+    const uint8_t *codes = second ? codes_w : codes_x;
+    uint8_t *out = second ? out_w : out_x;
+    const int bits = second ? bits_w : bits_x;
+    switch (bits == 1 ? 1 : bits == 2 ? 2 : bits <= 4 ? 4 : 8) {
+        case 1: unpack_group<1>(codes, bits, g, out, e2m1 != 0); break;
+        case 2: unpack_group<2>(codes, bits, g, out, e2m1 != 0); break;
+        case 4: unpack_group<4>(codes, bits, g, out, false); break;
+        default: unpack_group<8>(codes, bits, g, out, false); break;
+    }
+}
+
 // Row sums of an int8 matrix [rows x K]: one warp per row.
 __global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, int K, int32_t *__restrict__ out) {
     pdl_launch_dependents();
@@ -983,6 +1024,20 @@ int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_
     if (e != cudaSuccess) return cuda_fail(e);
     if (rowsum) return launch_rowsum(out, rows, K, rowsum, st);
     return QUEST_OK;
+}
+
+int launch_unpack_pair(const uint8_t *xq, int bits_x, int64_t M, int8_t *a8, int32_t *rs_a,
+                       const uint8_t *wq, int bits_w, int64_t N, int8_t *b8, int32_t *rs_b, int64_t K, bool e2m1,
+                       cudaStream_t st) {
+    const long long gx = M * K / 32, gw = N * K / 32;
+    if (gx + gw == 0) return QUEST_OK;
+    cudaError_t e = launch_pdl(unpack_pair_kernel, dim3((unsigned)((gx + gw + 127) / 128)), dim3(128), 0, st, 1, xq, bits_x, gx,
+                               reinterpret_cast<uint8_t *>(a8), wq, bits_w, gw, reinterpret_cast<uint8_t *>(b8), e2m1 ? 1 : 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int s = QUEST_OK;
+    if (rs_a) s = launch_rowsum(a8, M, K, rs_a, st);
+    if (!s && rs_b) s = launch_rowsum(b8, N, K, rs_b, st);
+    return s;
 }
 
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st) {

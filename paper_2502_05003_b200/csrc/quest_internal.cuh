@@ -117,6 +117,10 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                     float trust_factor, cudaStream_t st, int grid = GRID_UNIFORM);
 int launch_unpack(const uint8_t *codes, int bits, int64_t rows, int64_t K, int8_t *out,
                   int32_t *rowsum, cudaStream_t st, bool e2m1 = false);
+// Both operands of one contraction in a single launch (row sums follow where asked for).
+int launch_unpack_pair(const uint8_t *xq, int bits_x, int64_t M, int8_t *a8, int32_t *rs_a,
+                       const uint8_t *wq, int bits_w, int64_t N, int8_t *b8, int32_t *rs_b, int64_t K, bool e2m1,
+                       cudaStream_t st);
 int launch_rowsum(const int8_t *a8, int64_t rows, int64_t K, int32_t *rowsum, cudaStream_t st);
 int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b,
                 int bits_x, int bits_w, const float *sx, const float *sw,
