@@ -940,8 +940,8 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
             // the specialised tail: codes, scales and masks requested (or the rotation alone), trust_factor >= 1,
-            // below 8 bits; the FP4 grid has no separate GEMM operand
-            bool fast_tail = bits < 8 && trust_factor >= 1.0f && S >= 32;
+            // no row sums (so not the 8-bit GEMM operand); the FP4 grid has no separate GEMM operand
+            bool fast_tail = trust_factor >= 1.0f && S >= 32;
             for (int j = 0; j < 2; ++j) {
                 const QuantTensor &t = a.t[j];
                 const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
