@@ -195,7 +195,7 @@ int launch_hadamard_rows(const void *in, int in_dtype, int64_t ld_in, int64_t ro
     const int T = (int)(cols / 32);
     int S;
     if (T < 32) { S = 1; while (S < T) S <<= 1; } else { S = (T + 31) / 32 * 32; }
-    const int R = S >= 256 ? 1 : 256 / S;
+    const int R = S <= 128 ? 128 / S : 1;      // CTAs of 128 threads where a row fits
     const int threads = R * S;
     const size_t smem = had_block >= 2048 ? sizeof(float) * 32 * (size_t)threads : 0;
     if (smem > 48 * 1024) {
