@@ -193,8 +193,7 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // thread holds.  GFULL: had_block >= E, so every in-register stage runs.  FAST: the common case
 // fixed at compile time -- had_block = 128 with the first stage already applied, rows of at least
 // one warp, codes, scales and mask requested (the GEMM operand and the bfloat16 outputs of the
-// weight-only variant and the row sums of the 8-bit operand are optional; a tensor may also ask for the
-// rotation alone),
+// weight-only variant are optional; a tensor may also ask for the rotation alone), no row sums,
 // trust_factor >= 1 -- so that no per-row loop and only a few uniform branches remain.
 template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
@@ -465,7 +464,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                if (tn.rowsum) {
+                if (!FAST && tn.rowsum) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q) rsum += sum_bytes_s8(o[q]);
                 }
@@ -473,7 +472,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
             }
         }
     }
-    if (tn.rowsum) {                                   // uniform over the CTA
+    if (!FAST && tn.rowsum) {                                   // uniform over the CTA
         for (int m = 1; m < lanes_per_row; m <<= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, m);
         if (S > 32) {
             int *ism = reinterpret_cast<int *>(xsm);
@@ -940,13 +939,13 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             a.inv_sqrt_g = 1.0f / sqrtf((float)had_block);
             const dim3 grid((unsigned)(nb[0] + nb[1]));
             cudaError_t e;
-            // the specialised tail: codes, scales and masks requested (or the rotation alone), trust_factor >= 1;
-            // the FP4 grid has no separate GEMM operand
+            // the specialised tail: codes, scales and masks requested (or the rotation alone), trust_factor >= 1,
+            // no row sums (so not the 8-bit GEMM operand); the FP4 grid has no separate GEMM operand
             bool fast_tail = trust_factor >= 1.0f && S >= 32;
             for (int j = 0; j < 2; ++j) {
                 const QuantTensor &t = a.t[j];
                 const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
-                if (t.rows > 0 && !((t.codes && t.scales && t.mask) || rot_only)) fast_tail = false;
+                if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fast_tail = false;
                 if (t.rows > 0 && grid_kind == GRID_FP4 && (t.op8 || t.rot || t.cbf)) fast_tail = false;
             }
             int dev = 0, sms = 148;
