@@ -195,7 +195,7 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // one warp, codes, scales and mask requested (the GEMM operand and the bfloat16 outputs of the
 // weight-only variant are optional; a tensor may also ask for the rotation alone), no row sums,
 // trust_factor >= 1 -- so that no per-row loop and only a few uniform branches remain.
-template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false>
+template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false, bool RS = false>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
                                                      int s_start) {
@@ -464,7 +464,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
                 uint4 *dst = reinterpret_cast<uint4 *>(tn.op8 + row * (long long)cols + (long long)tr * E + g32 * 32);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                if (!FAST && tn.rowsum) {
+                if ((RS || !FAST) && tn.rowsum) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q) rsum += sum_bytes_s8(o[q]);
                 }
@@ -472,7 +472,7 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
             }
         }
     }
-    if (!FAST && tn.rowsum) {                                   // uniform over the CTA
+    if ((RS || !FAST) && tn.rowsum) {                                   // uniform over the CTA
         for (int m = 1; m < lanes_per_row; m <<= 1) rsum += __shfl_xor_sync(0xffffffffu, rsum, m);
         if (S > 32) {
             int *ism = reinterpret_cast<int *>(xsm);
@@ -777,7 +777,8 @@ static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaS
 // one CTA per row group: at sizes whose whole input is a few waves of CTAs the hardware's own CTA
 // scheduling balances better than the persistent loop of the streaming kernel and there is no
 // staging to set up.  Stride 64 pairs this thread with lane ^ 2 (shuffles); the rest is the common tail.
-template <int CB, int GRID = GRID_UNIFORM>
+// RS: the row sums of the 8-bit GEMM operand are wanted (kept out of the common instantiation).
+template <int CB, int GRID = GRID_UNIFORM, bool RS = false>
 __global__ void __launch_bounds__(256, 4)
 quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
     extern __shared__ float xsm[];                 // [warps] partial sums
@@ -817,11 +818,13 @@ quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
             v[i] = __ffma2_rn(v[i], sgn, p);
         }
     }
-    rotate_project_store<CB, 32, true, true, GRID>(v, a, tn, active, row, tr, r_local, xsm, 32);
+    rotate_project_store<CB, 32, true, true, GRID, false, RS>(v, a, tn, active, row, tr, r_local, xsm, 32);
 }
 
 template <int GRID>
-static cudaError_t launch_direct128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
+static cudaError_t launch_direct128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                                    bool rowsums = false) {
+    if (rowsums) return launch_pdl(quantize_direct128_kernel<8, GRID_UNIFORM, true>, grid, dim3(threads), smem, st, 1, a);
     if (GRID == GRID_FP4) return launch_pdl(quantize_direct128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
     switch (cb) {
         case 1: return launch_pdl(quantize_direct128_kernel<1, GRID>, grid, dim3(threads), smem, st, 1, a);
@@ -942,10 +945,13 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             // the specialised tail: codes, scales and masks requested (or the rotation alone), trust_factor >= 1,
             // no row sums (so not the 8-bit GEMM operand); the FP4 grid has no separate GEMM operand
             bool fast_tail = trust_factor >= 1.0f && S >= 32;
+            bool fast_tail_rs = fast_tail, any_rowsum = false;   // the same with row sums allowed
             for (int j = 0; j < 2; ++j) {
                 const QuantTensor &t = a.t[j];
                 const bool rot_only = t.rot && !t.codes && !t.scales && !t.mask && !t.op8 && !t.cbf;
                 if (t.rows > 0 && (t.rowsum || !((t.codes && t.scales && t.mask) || rot_only))) fast_tail = false;
+                if (t.rows > 0 && !((t.codes && t.scales && t.mask) || rot_only)) fast_tail_rs = false;
+                if (t.rows > 0 && t.rowsum) any_rowsum = true;
                 if (t.rows > 0 && grid_kind == GRID_FP4 && (t.op8 || t.rot || t.cbf)) fast_tail = false;
             }
             int dev = 0, sms = 148;
@@ -963,6 +969,9 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                 else
                     e = fast_tail ? launch_wide<GRID_UNIFORM, true>(cb, g, threads, smem2, st, a, exchange)
                                   : launch_wide<GRID_UNIFORM, false>(cb, g, threads, smem2, st, a, exchange);
+            } else if (e32 && had_block == 128 && fast_tail_rs && any_rowsum && cb == 8 && grid_kind == GRID_UNIFORM && threads <= 256) {
+                // 8-bit codes with the row sums the GEMM needs
+                e = launch_direct128<GRID_UNIFORM>(cb, grid, threads, smem, st, a, true);
             } else if (e32 && had_block == 128 && fast_tail && threads <= 256) {
                 // the common case: direct loads, one CTA per row group
                 e = grid_kind == GRID_FP4 ? launch_direct128<GRID_FP4>(cb, grid, threads, smem, st, a)
