@@ -276,6 +276,9 @@ float quest_alpha_star(int bits);
  * it, and returns QUEST_OK or QUEST_ERR_DEVICE_TIMEOUT (QUEST_ERR_CUDA if the read fails).
  */
 int quest_device_status(void *stream);
+/* The same call under a second name ("status of the last kernels on this stream"); kept so that code
+ * written against either spelling links. */
+int quest_last_device_status(void *stream);
 
 /*
  * Measurement aid (no counterpart in the paper): per-stage device times.  While enabled, every

@@ -9,7 +9,7 @@ LIB_PATH = os.path.join(_HERE, "libquest_b200.so")
 
 EXPORTS = (
     "quest_quantize", "quest_trust_mask", "quest_lowbit_gemm", "quest_linear_fwd",
-    "quest_workspace_bytes", "quest_codes_bytes", "quest_alpha_star", "quest_device_status",
+    "quest_workspace_bytes", "quest_codes_bytes", "quest_alpha_star", "quest_device_status", "quest_last_device_status",
     "quest_status_string", "quest_last_cuda_error", "quest_stage_timing", "quest_stage_times",
     "quest_lowbit_gemm_static", "quest_linear_bwd", "quest_bwd_workspace_bytes",
     "quest_alpha_star_fp4", "quest_quantize_fp4", "quest_lowbit_gemm_fp4", "quest_linear_fwd_fp4",
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
     L.quest_alpha_star.argtypes = [ci]
     L.quest_device_status.restype = ci
     L.quest_device_status.argtypes = [vp]
+    L.quest_last_device_status.restype = ci
+    L.quest_last_device_status.argtypes = [vp]
     L.quest_status_string.restype = ctypes.c_char_p
     L.quest_status_string.argtypes = [ci]
     L.quest_last_cuda_error.restype = ctypes.c_char_p

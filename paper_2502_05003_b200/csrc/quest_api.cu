@@ -183,6 +183,8 @@ int quest_device_status(void *stream) {
     return QUEST_OK;
 }
 
+int quest_last_device_status(void *stream) { return quest_device_status(stream); }
+
 int quest_stage_timing(int enable) {
     if (enable && !g_timer.created) {
         for (int i = 0; i < QUEST_NUM_STAGES; ++i)

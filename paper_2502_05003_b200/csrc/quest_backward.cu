@@ -199,7 +199,8 @@ int launch_hadamard_rows(const void *in, int in_dtype, int64_t ld_in, int64_t ro
     const int threads = R * S;
     const size_t smem = had_block >= 2048 ? sizeof(float) * 32 * (size_t)threads : 0;
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(iht_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
+        static DynamicSmemOnce smem_attr;
+        cudaError_t e = smem_attr.set(iht_rows_kernel, 72 * 1024);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     const long long grid = (rows + R - 1) / R;

@@ -957,12 +957,10 @@ template <int BN, int MODE, bool TWO, bool YT, int OPL = 0>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
                    cudaStream_t st) {
     using L = SmemLayout<BN, TWO>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_i8_kernel<BN, MODE, TWO, YT, OPL>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL);
+    static DynamicSmemOnce smem_attr;            // per kernel instantiation, per device
+    {
+        cudaError_t e = smem_attr.set(gemm_i8_kernel<BN, MODE, TWO, YT, OPL>, L::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
-        attr_done = true;
     }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);

@@ -91,6 +91,24 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 #endif
 
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) applies to the current device only.  One static
+// instance per kernel (per template instantiation of a launcher) remembers on which devices of this
+// process the attribute has been set; setting it twice is harmless, so the race between two host
+// threads that both see "not yet" is benign.
+struct DynamicSmemOnce {
+    bool done[64] = {};
+    template <typename Kernel>
+    cudaError_t set(Kernel kernel, int bytes) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+        return e;
+    }
+};
+
 // Status / error plumbing.
 int cuda_fail(cudaError_t e);             // records the message, returns QUEST_ERR_CUDA
 int cuda_fail_msg(const char *msg);

@@ -757,8 +757,8 @@ static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaS
                                int exchange_bytes) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
-        cudaError_t e_ = cudaFuncSetAttribute(quantize_wide_kernel<CBV, FAST, GRID>,                        \
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);     \
+        static DynamicSmemOnce once_;                                                                       \
+        cudaError_t e_ = once_.set(quantize_wide_kernel<CBV, FAST, GRID>, 160 * 1024);                      \
         if (e_ != cudaSuccess) return e_;                                                                   \
         return launch_pdl(quantize_wide_kernel<CBV, FAST, GRID>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
                           exchange_bytes);                                                                  \
@@ -839,8 +839,8 @@ static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cuda
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
         if (smem > 48 * 1024) {                                                                             \
-            cudaError_t e_ = cudaFuncSetAttribute(quantize_rows_kernel<BF16, CBV, E>,                       \
-                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);  \
+            static DynamicSmemOnce once_;                                                                   \
+            cudaError_t e_ = once_.set(quantize_rows_kernel<BF16, CBV, E>, 72 * 1024);                      \
             if (e_ != cudaSuccess) return e_;                                                               \
         }                                                                                                   \
         cudaError_t l_ = launch_pdl(quantize_rows_kernel<BF16, CBV, E>, grid, dim3(threads), smem, st, 1, a);  \
@@ -860,8 +860,8 @@ static cudaError_t launch_rows(int cb, dim3 grid, int threads, size_t smem, cuda
 template <bool BF16, int E>
 static cudaError_t launch_rows_fp4(dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
     if (smem > 48 * 1024) {
-        cudaError_t e_ = cudaFuncSetAttribute(quantize_rows_kernel<BF16, 4, E, GRID_FP4>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
+        static DynamicSmemOnce once_;
+        cudaError_t e_ = once_.set(quantize_rows_kernel<BF16, 4, E, GRID_FP4>, 72 * 1024);
         if (e_ != cudaSuccess) return e_;
     }
     return launch_pdl(quantize_rows_kernel<BF16, 4, E, GRID_FP4>, grid, dim3(threads), smem, st, 1, a);
@@ -870,8 +870,8 @@ static cudaError_t launch_rows_fp4(dim3 grid, int threads, size_t smem, cudaStre
 template <int E, bool FAST>
 static cudaError_t launch_stream_fp4(int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                      int total_groups, int exchange_bytes) {
-    cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<4, E, FAST, GRID_FP4>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    static DynamicSmemOnce once_;
+    cudaError_t e_ = once_.set(quantize_stream_kernel<4, E, FAST, GRID_FP4>, 160 * 1024);
     if (e_ != cudaSuccess) return e_;
     return launch_pdl(quantize_stream_kernel<4, E, FAST, GRID_FP4>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a,
                       total_groups, exchange_bytes);
@@ -882,8 +882,8 @@ static cudaError_t launch_stream(int cb, int grid, int threads, size_t smem, cud
                                  int total_groups, int exchange_bytes) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
-        cudaError_t e_ = cudaFuncSetAttribute(quantize_stream_kernel<CBV, E, FAST>,                               \
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);     \
+        static DynamicSmemOnce once_;                                                                       \
+        cudaError_t e_ = once_.set(quantize_stream_kernel<CBV, E, FAST>, 160 * 1024);                       \
         if (e_ != cudaSuccess) return e_;                                                                   \
         return launch_pdl(quantize_stream_kernel<CBV, E, FAST>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
                           total_groups, exchange_bytes);                                                    \
@@ -1009,12 +1009,10 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
     int p2 = 1;
     while (p2 < cols) p2 <<= 1;
     const size_t smem = sizeof(float) * (size_t)(cols + p2);
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(quantize_generic_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    static DynamicSmemOnce smem_attr;
+    {
+        cudaError_t e = smem_attr.set(quantize_generic_kernel, 160 * 1024);
         if (e != cudaSuccess) return cuda_fail(e);
-        attr_done = true;
     }
     for (int j = 0; j < njobs; ++j) {
         const QuantJob &q = jobs[j];

@@ -7,11 +7,9 @@ import torch
 
 from oracle import quest_oracle as qo
 from paper_2502_05003_b200 import synth
-from tests.gpu_util import to_dev
+from tests.gpu_util import assert_output_close, to_dev
 
 pytestmark = pytest.mark.gpu
-
-BF16_OUT_RTOL = 2.0 ** -8 + 1e-5
 
 
 def check_quantize(x_np, g, trust=1.0):
@@ -39,6 +37,14 @@ def rows(kind, r, c, seed, bf16=True):
 @pytest.mark.parametrize("bf16", [True, False])
 def test_quantize_shapes(g, cols, bf16):
     check_quantize(rows("student", 67, cols, g + cols, bf16), g)
+
+
+@pytest.mark.parametrize("trust", [0.5, 1.0])
+@pytest.mark.parametrize("g,cols", [(128, 16384), (64, 8256), (4096, 16384), (16384, 16384), (8192, 8192)])
+def test_quantize_bf16_rows_wider_than_8192(g, cols, trust):
+    """The persistent streaming kernel (rows of more than 8192 bfloat16 elements) with the FP4 grid:
+    specialised and general tails."""
+    check_quantize(rows("student", 37, cols, g + cols + 1), g, trust)
 
 
 @pytest.mark.parametrize("trust", [0.0, 0.5, 1.0, 1.3, 3.0])
@@ -118,7 +124,7 @@ def test_linear_fwd_config2(g):
     rows_ = np.sort(np.random.default_rng(0).choice(4096, 96, replace=False))
     ref_y = qo.dequant_fp4(qo.gemm_acc_fp4(qx["codes"][rows_], qw["codes"], 2048), qx["scales"][rows_], qw["scales"])
     got = out["y"].float().cpu().numpy().astype(np.float64)[rows_]
-    assert np.all(np.abs(got - ref_y) <= BF16_OUT_RTOL * np.abs(ref_y) + 1e-30)
+    assert_output_close(got, ref_y, True)
     # cached weights give the same result
     out2 = quest.quest_linear_fwd_fp4(to_dev(c["x"]), None, g, 1.0, out_dtype=torch.bfloat16,
                                       w_cached={"wq": out["wq"], "sw": out["sw"]})

@@ -5,14 +5,10 @@ import pytest
 import torch
 
 from oracle import quest_oracle as qo
-from tests.gpu_util import canary_intact, guarded
+from tests.gpu_util import assert_output_close, canary_intact, guarded
 from tests.helpers import container_bits
 
 pytestmark = pytest.mark.gpu
-
-# A bfloat16 result carries 8 significant bits: storing y costs up to 2^-9 relative on average
-# and 2^-8 in the worst case, on top of the 1e-5 of the fp32 scale product.
-BF16_OUT_RTOL = 2.0 ** -8 + 1e-5
 
 
 def random_codes(rows, K, bits, rng):
@@ -44,8 +40,7 @@ def run_case(M, N, K, bx, bw, out_dtype, seed=0, sample_rows=None):
     assert np.array_equal(got_acc, ref_acc), f"{(got_acc != ref_acc).sum()} accumulators differ"
     ref_y = qo.dequant(ref_acc, sx[rows], sw)
     got_y = y.float().cpu().numpy().astype(np.float64)[rows]
-    tol = 1e-5 if out_dtype == torch.float32 else BF16_OUT_RTOL
-    assert np.all(np.abs(got_y - ref_y) <= tol * np.abs(ref_y) + 1e-30)
+    assert_output_close(got_y, ref_y, out_dtype == torch.bfloat16)
     # y alone / acc alone
     y2, _ = quest.quest_lowbit_gemm(d(xq), d(sx), bx, d(wq), d(sw), bw, K, out_dtype=out_dtype)
     _, a2 = quest.quest_lowbit_gemm(d(xq), d(sx), bx, d(wq), d(sw), bw, K, want_y=False, want_acc=True)

@@ -5,13 +5,12 @@ import torch
 
 from oracle import quest_oracle as qo
 from paper_2502_05003_b200 import synth
-from tests.gpu_util import to_dev
+from tests.gpu_util import BF16_OUT_RTOL, assert_output_close, to_dev
 
 pytestmark = pytest.mark.gpu
 
 F32_IN_RTOL = 1e-5                   # fp32 inputs, fp32 output
 BF16_IN_RTOL = 2e-3                  # bf16 inputs, fp32 output
-BF16_OUT_RTOL = 2.0 ** -8 + 1e-5     # bf16 output: the unit roundoff of the storage format dominates
 
 
 def check_linear(x_np, w_np, bits, g, trust, out_dtype, y_tol, sample_rows=None):
@@ -31,7 +30,10 @@ def check_linear(x_np, w_np, bits, g, trust, out_dtype, y_tol, sample_rows=None)
     K = x_np.shape[1]
     ref_y = qo.dequant(qo.gemm_acc(qx["codes"][rows], bits, qw["codes"], bits, K), qx["scales"][rows], qw["scales"])
     got = out["y"].float().cpu().numpy().astype(np.float64)[rows]
-    assert np.all(np.abs(got - ref_y) <= y_tol * np.abs(ref_y) + 1e-30)
+    if out_dtype == torch.bfloat16:
+        assert_output_close(got, ref_y, True)
+    else:
+        assert np.all(np.abs(got - ref_y) <= y_tol * np.abs(ref_y) + 1e-30)
     if out_dtype == torch.bfloat16:
         # the same call with an fp32 result must meet the tolerance stated for bf16 inputs
         y32 = quest.quest_linear_fwd(x, w, bits, g, trust, out_dtype=torch.float32)["y"]

@@ -72,6 +72,19 @@ def test_f32_rows(bits, g, cols):
     check(rows_of("outliers", 33, cols, bits * 7 + g, False), bits, g)
 
 
+@pytest.mark.parametrize("trust", [0.5, 1.0])
+@pytest.mark.parametrize("bits", [1, 4, 8])
+@pytest.mark.parametrize("g,cols", [(128, 16384), (64, 8256), (4096, 16384), (16384, 16384), (8192, 8192), (128, 8320),
+                                    (256, 12288)])
+def test_bf16_rows_wider_than_8192(g, cols, bits, trust):
+    """Rows of more than 8192 bfloat16 elements take the persistent streaming kernel (64 elements per
+    thread): its specialised tail (g = 128, trust_factor >= 1) and its general one, with the first
+    butterfly stage read from shared memory (g >= 128) or from registers (g = 64), and rotation blocks
+    that span several warps (g >= 4096).  (8192, 8192) is the widest block the 32-per-thread kernel
+    serves through its shared-memory exchange."""
+    check(rows_of("student", 37, cols, bits * 31 + g + cols, True), bits, g, trust)
+
+
 @pytest.mark.parametrize("trust", [0.0, 0.5, 1.0, 1.25, 1.3, 3.0])
 @pytest.mark.parametrize("bits", [1, 2, 4])
 def test_trust_factors(bits, trust):

@@ -4,10 +4,12 @@ Some users of this library only ever hold the pointers they are given: a plug-in
 application, or a server whose own pools took all of device memory at start-up, so a later
 cudaMalloc for a workspace fails.  For them the library keeps the GEMM's scratch in a fixed
 array of its own.  These tests call that entry point through the C ABI with every output
-preallocated and check it against ``quest_lowbit_gemm`` (which takes a caller-made workspace):
-int32 accumulators bit for bit, outputs within the tolerance the other GEMM tests use.  Two calls
-run back to back with different shapes and bit-widths, because the array is shared and keeps the
-previous call's bytes.  The file sorts last so that a run stopping at the first failure has
+preallocated and check it against the CPU oracle (int32 accumulators bit for bit, outputs within the
+tolerance the other GEMM tests use) and against ``quest_lowbit_gemm``, which takes a caller-made
+workspace.  The call is also watched for allocations: the free device memory the driver reports and
+the bytes torch's allocator holds must both be the same after it as before.  Several calls run back to
+back with different shapes and bit-widths, because the array is shared and keeps the previous
+call's bytes.  The file sorts last so that a run stopping at the first failure has
 already run every other test; it passes alone in a fresh process as well.
 """
 import ctypes
@@ -17,8 +19,6 @@ import pytest
 import torch
 
 from tests.helpers import container_bits
-
-BF16_OUT_RTOL = 2.0 ** -8 + 1e-5     # as in tests/test_gpu_gemm.py
 
 
 def _random_codes(rows, K, bits, rng):
@@ -42,18 +42,36 @@ def _one_call(quest, M, N, K, bx, bw, out_dtype, seed):
     # outputs of the static variant are made here, by the caller, before the call
     y = torch.full((M, N), float("nan"), dtype=out_dtype, device="cuda")
     acc = torch.full((M, N), -1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    free_before, held_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_reserved()
     quest.quest_lowbit_gemm_static(xq, sx, bx, wq, sw, bw, K, y=y, acc=acc)
     torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
+    assert torch.cuda.memory_reserved() == held_before, "the call went through torch's allocator"
     assert quest.quest_device_status() == 0
+    # the oracle decides: exact integer contraction of the same codes, then the scale product
+    from oracle import quest_oracle as qo
+    from tests.gpu_util import assert_output_close
+    codes_x, codes_w = xq.cpu().numpy(), wq.cpu().numpy()
+    ref_acc = qo.gemm_acc(codes_x, bx, codes_w, bw, K)
+    assert np.array_equal(acc.cpu().numpy(), ref_acc), "int32 accumulators differ from the oracle"
+    ref_y = qo.dequant(ref_acc, sx.cpu().numpy(), sw.cpu().numpy())
+    assert_output_close(y.double().cpu().numpy(), ref_y, out_dtype == torch.bfloat16)
+    # and the two entry points agree with each other bit for bit (same kernels, different scratch)
     assert torch.equal(acc, acc_ref), "int32 accumulators differ from quest_lowbit_gemm"
-    got, ref = y.double(), y_ref.double()
-    tol = 1e-5 if out_dtype == torch.float32 else BF16_OUT_RTOL
-    assert bool((torch.abs(got - ref) <= tol * torch.abs(ref) + 1e-30).all())
+    assert torch.equal(y, y_ref), "outputs differ from quest_lowbit_gemm"
 
 
 @pytest.mark.gpu
 def test_static_scratch_matches_workspace_variant_on_two_calls_in_a_row():
     import paper_2502_05003_b200 as quest
+    # The first call on a device looks the array's address up, and the CUDA runtime may only then load
+    # the part of the library image that holds it; that one-time set-up is documented and is kept out
+    # of the allocation watch by making it here, on a tiny problem.
+    tiny = torch.zeros((8, 16), dtype=torch.uint8, device="cuda")
+    one = torch.ones(8, device="cuda")
+    quest.quest_lowbit_gemm_static(tiny, one, 4, tiny, one, 4, 32, acc=torch.empty((8, 8), dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
     # first call nearly fills the array ((M + N) * K = 3.9 Mi bytes of int8 operands) ...
     _one_call(quest, 1000, 900, 2048, 4, 4, torch.bfloat16, seed=11)
     # ... the second is smaller, ragged and uses 8-bit codes (row sums live in the same array),
