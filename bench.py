@@ -2,14 +2,17 @@
 """Benchmark of the QuEST quantized-linear forward hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--had-block G]
-                    [--no-graph] [--pass backward|weight_only] [--bits B]
+                    [--no-graph] [--pass backward|weight_only] [--bits B] [--no-config4]
 
 One "step" is one pass of the whole path (Algorithm 1: quantize X, quantize W, low-bit GEMM with
 the dequantising epilogue) through the C ABI call ``quest_linear_fwd`` on the 1.6B-scale layer:
 X[4096 x 2048] bf16, W[2048 x 2048] bf16, b = 4, Hadamard block 128 (seeded synthetic data).
-The step rotates over a ring of buffer sets larger than L2, so every step streams from HBM, and the
-timed steps are replayed from a CUDA graph holding one pass over the ring (``--no-graph``: direct
-launches), because the host cannot launch a step of a few tens of microseconds fast enough.
+The step rotates over a ring of buffer sets larger than L2, so every step streams from HBM.  The K
+timed steps are replayed from a CUDA graph whose length divides K (``--no-graph``: direct launches),
+because the host cannot launch a step of a few tens of microseconds fast enough.  The block of K
+steps is timed at least 20 times (and until a quarter of a second of device time has accumulated),
+each time bracketed by a barrier and a device synchronisation on both sides; the line reports the
+median block, with the fastest and slowest beside it.
 ``--pass backward`` times Algorithm 2 (``quest_linear_bwd``) on the same layer instead, and
 ``--pass weight_only`` the weight-only forward of Section 4.5 (``quest_linear_fwd_weight_only``).
 
@@ -24,6 +27,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -39,12 +43,12 @@ TOKENS, HIDDEN, OUT, BITS = 4096, 2048, 2048, 4
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 : dense bf16 tensor throughput (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from one ncu capture of this command's
-# kernels (None when no capture of the current kernel exists).
-GEMM_DRAM_TRAFFIC_BYTES = 12652032          # low-bit GEMM, 4096 x 2048 x 2048
-QUANT_DRAM_TRAFFIC_BYTES = 25191168         # quantizer, x and w in one launch
-QUANT_INSTR_PER_ELEMENT = 23.3              # thread instructions per element, same capture
+COUNTERS_FILE = os.path.join(ROOT, "profiles", "ncu_counters.txt")
+MIN_REPETITIONS = 20                  # the timed block of K steps is repeated at least this often ...
+MIN_TIMED_SECONDS = 0.25              # ... and until this much device time has accumulated
+MAX_REPETITIONS = 1000
+MAX_GRAPH_STEPS = 256
+BRACKETED = "event nodes around the kernel, no programmatic overlap with its neighbours (an upper bound)"
 
 
 def load_peaks():
@@ -57,6 +61,19 @@ def load_peaks():
     p = dict(FALLBACK_PEAKS)
     p["_source"] = "fallback"
     return p
+
+
+def load_ncu_counters() -> dict:
+    """Counters of one ncu capture per kernel, written by ``python -m paper_2502_05003_b200.ncu_counters``
+    into profiles/ncu_counters.txt together with a hash of the kernel sources they were taken from.
+    A kernel whose sources have changed since reports no counters at all, never stale ones."""
+    if not os.path.exists(COUNTERS_FILE):
+        return {}
+    try:
+        from paper_2502_05003_b200 import ncu_counters
+        return ncu_counters.read(COUNTERS_FILE, only_current=True)
+    except Exception:
+        return {}
 
 
 def workload_config(had_block: int) -> dict:
@@ -78,7 +95,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
     def __init__(self, device_index: int, period_s: float = 0.002):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.stamps, self.reasons, self.max_mhz = [], [], set(), None
         self._stop = threading.Event()
         self._thread = None
         self._idx, self._period = device_index, period_s
@@ -102,6 +119,7 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                self.stamps.append(time.perf_counter())
                 mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
                 for k, bit in names.items():
                     if mask & bit:
@@ -121,10 +139,18 @@ class ClockSampler:
         if self._thread is not None:
             self._thread.join()
 
+    def nearest(self, t: float):
+        """SM clock of the sample taken closest to host time t (None without samples)."""
+        if not self.stamps:
+            return None
+        i = min(range(len(self.stamps)), key=lambda j: abs(self.stamps[j] - t))
+        return self.samples[i]
+
     def summary(self) -> dict:
         s = sorted(self.samples)
         med = s[len(s) // 2] if s else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s),
+                "sm_mhz_min": s[0] if s else None}
 
 
 # ------------------------------------------------------------------------------------ ranks
@@ -136,20 +162,44 @@ def init_ranks(n_gpus: int):
     return rank, world, local
 
 
-def max_over_ranks(value: float, world: int, backend_device=None) -> float:
-    """Max of a scalar over all ranks (identity at world size 1)."""
+def max_over_ranks(value, world: int, backend_device=None):
+    """Element-wise max of a scalar or a list of scalars over all ranks (identity at world size 1)."""
     if world <= 1:
         return value
     import torch
     import torch.distributed as dist
-    t = torch.tensor([value], dtype=torch.float64, device=backend_device or "cpu")
+    scalar = not isinstance(value, (list, tuple))
+    t = torch.tensor([value] if scalar else list(value), dtype=torch.float64, device=backend_device or "cpu")
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
+    return float(t[0].item()) if scalar else [float(v) for v in t.tolist()]
 
 
 def aggregate_tokens_per_s(tokens_per_rank_step: int, steps: int, world: int, max_elapsed_s: float) -> float:
     """Whole-job throughput of independent replicas: all ranks' tokens over the slowest rank's time."""
     return tokens_per_rank_step * steps * world / max_elapsed_s
+
+
+def median(values):
+    s = sorted(values)
+    n = len(s)
+    return s[n // 2] if n % 2 else 0.5 * (s[n // 2 - 1] + s[n // 2])
+
+
+def repetition_count(pilot_seconds: float, min_reps: int = MIN_REPETITIONS) -> int:
+    """How often the timed block is repeated: at least `min_reps`, and enough for MIN_TIMED_SECONDS."""
+    want = int(math.ceil(MIN_TIMED_SECONDS / max(pilot_seconds, 1e-9)))
+    return max(min_reps, min(MAX_REPETITIONS, want))
+
+
+def graph_length(steps: int, n_sets: int) -> int:
+    """Steps held by the captured graph: a divisor of `steps`, so that the timed block is whole replays
+    and nothing is launched directly; at least one pass over the ring where a divisor allows it."""
+    if steps <= MAX_GRAPH_STEPS:
+        return steps
+    for g in range(MAX_GRAPH_STEPS, 0, -1):
+        if steps % g == 0 and g >= n_sets:
+            return g
+    return steps
 
 
 # ------------------------------------------------------------------------------------ oracle legs
@@ -215,6 +265,235 @@ def run_reference(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------ timing helpers
+
+class Stepper:
+    """Runs `step(i)` for i = 0, 1, ... either directly or by replaying a CUDA graph that holds
+    `graph_length(k)` consecutive steps (the steps cycle over the caller's ring of buffer sets)."""
+
+    def __init__(self, step, n_sets: int, dev, no_graph: bool):
+        import torch
+        self.torch, self.step, self.n_sets, self.dev, self.no_graph = torch, step, n_sets, dev, no_graph
+        self.side = torch.cuda.Stream(device=dev)
+        self.graphs = {}
+
+    def graph_for(self, length: int):
+        torch = self.torch
+        if length not in self.graphs:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(self.side):
+                for i in range(min(length, self.n_sets)):        # warm every kernel outside the capture
+                    self.step(i)
+                self.side.synchronize()
+                with torch.cuda.graph(g, stream=self.side):
+                    for i in range(length):
+                        self.step(i)
+            torch.cuda.synchronize()
+            self.graphs[length] = g
+        return self.graphs[length]
+
+    def prepare(self, k: int):
+        if not self.no_graph:
+            self.graph_for(graph_length(k, self.n_sets))
+
+    def run(self, k: int):
+        if self.no_graph:
+            for i in range(k):
+                self.step(i)
+            return
+        length = graph_length(k, self.n_sets)
+        g = self.graph_for(length)
+        for _ in range(k // length):
+            g.replay()
+
+    def launch_mode(self, k: int) -> str:
+        if self.no_graph:
+            return "direct"
+        length = graph_length(k, self.n_sets)
+        return f"CUDA graph of {length} steps x {k // length} replays, no direct launches"
+
+
+def timed_repetitions(stepper: Stepper, k: int, barrier, world: int, dev, local: int, min_reps: int = MIN_REPETITIONS):
+    """Times the block of k steps repeatedly; every repetition is bracketed by barrier + synchronize
+    on both sides and timed with CUDA events on the launching stream.  Returns (seconds per
+    repetition, max over ranks; the clock sampler; the nearest SM clock sample of each repetition)."""
+    import torch
+    stepper.prepare(k)
+    stepper.run(k)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def one():
+        barrier()
+        e0.record()
+        stepper.run(k)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3
+
+    pilot = max_over_ranks(one(), world, dev)
+    reps = repetition_count(pilot, min_reps)
+    times, host_mid = [], []
+    with ClockSampler(local) as clocks:
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            times.append(one())
+            host_mid.append(0.5 * (t0 + time.perf_counter()))
+    barrier()
+    times = max_over_ranks(times, world, dev)
+    mhz = [clocks.nearest(t) for t in host_mid]
+    return times, clocks, mhz
+
+
+def spread(times, k: int, mhz=None) -> dict:
+    med = median(times)
+    out = {"n": len(times), "ms_per_step_median": 1e3 * med / k, "ms_per_step_min": 1e3 * min(times) / k,
+           "ms_per_step_max": 1e3 * max(times) / k}
+    if mhz and all(m is not None for m in mhz):
+        s = sorted(mhz)
+        out["sm_mhz_nearest_sample"] = {"min": s[0], "median": s[len(s) // 2], "max": s[-1]}
+        # time x clock, so that blocks run at different clocks can be compared
+        out["us_per_step_x_ghz_median"] = median([1e6 * t / k * m * 1e-3 for t, m in zip(times, mhz)])
+    return out
+
+
+def stage_times(quest, stepper: Stepper, n_sets: int, reps: int = 50) -> dict:
+    """Per-kernel durations: the same steps with every stage bracketed by CUDA events on the launching
+    stream.  Inside a graph the event records are graph nodes, so the host's launch rate does not sit
+    between an event and its kernel; each replay yields the stage times of the graph's last step.
+    A bracketed kernel cannot overlap its neighbours (programmatic dependent launch is cut by the
+    event nodes), so these durations are upper bounds of what each kernel costs inside the step."""
+    import torch
+    quest.quest_stage_timing(True)
+    quest.quest_stage_times(reset=2)
+    staged = None if stepper.no_graph else Stepper(stepper.step, n_sets, stepper.dev, False).graph_for(n_sets)
+    for r in range(reps):
+        if staged is None:
+            stepper.step(r)
+        else:
+            staged.replay()
+        quest.quest_stage_times()
+    stage = quest.quest_stage_times(reset=2)
+    quest.quest_stage_timing(False)
+    torch.cuda.synchronize()
+    return {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+
+
+def bracket_overhead_ms(dev, reps: int = 50):
+    """What two event nodes around a kernel node cost by themselves: the same bracket around a kernel
+    that does nothing measurable (a one-element fill), replayed from a graph.  Reported beside the
+    stage times; not subtracted from them."""
+    import torch
+    try:
+        a, b = torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True)
+        x = torch.zeros(1, device=dev)
+        st = torch.cuda.Stream(device=dev)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(st):
+            x.fill_(1.0)
+            st.synchronize()
+            with torch.cuda.graph(g, stream=st):
+                x.fill_(0.0)
+                a.record(st)
+                x.fill_(1.0)
+                b.record(st)
+        tot = 0.0
+        for _ in range(reps):
+            g.replay()
+            torch.cuda.synchronize()
+            tot += a.elapsed_time(b)
+        return tot / reps
+    except Exception:
+        return None
+
+
+def library_int8_tops(dev, m: int, n: int, k: int, iters: int = 20):
+    """The library's int8 GEMM (torch._int_mm -> cuBLASLt), timed only: a measured tensor-pipe reference."""
+    import torch
+    try:
+        a8 = torch.randint(-8, 8, (m, k), dtype=torch.int8, device=dev)
+        b8 = torch.randint(-8, 8, (k, n), dtype=torch.int8, device=dev)
+        for _ in range(3):
+            torch._int_mm(a8, b8)
+        torch.cuda.synchronize()
+        best = None
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                torch._int_mm(a8, b8)
+            e1.record()
+            torch.cuda.synchronize()
+            t = e0.elapsed_time(e1) * 1e-3 / iters
+            best = t if best is None else min(best, t)
+        return 2.0 * m * n * k / best / 1e12
+    except Exception:
+        return None
+
+
+# ------------------------------------------------------------------------------------ config 4
+
+def run_config4(quest, dev, peaks, int8_peaks: dict, no_graph: bool) -> dict:
+    """The Llama-style MLP block at 1.6B scale (config 4): X[8192 x 2048], gate/up W[5504 x 2048], down
+    W[2048 x 5504], b = 4, g = 128, every GEMM input quantized, SwiGLU between.  One buffer set: the
+    block touches several times L2 per pass.  Reports each layer's GEMM and quantizer against their
+    rooflines (event-bracketed stages) and the whole block replayed from one graph."""
+    import torch
+    from paper_2502_05003_b200 import synth
+    cfg = synth.config4()
+    T, H, I = 8192, 2048, 5504
+    t = lambda k: torch.from_numpy(cfg[k]).view(torch.bfloat16).to(dev)
+    x, wg, wu, wd = t("x"), t("w_gate"), t("w_up"), t("w_down")
+    sync = lambda: torch.cuda.synchronize()
+    local = dev.index or 0
+    bufs = quest.mlp_buffers(T, H, I, BITS, dev)
+
+    def block(_i=0):
+        quest.quest_mlp_fwd(x, wg, wu, wd, BITS, 128, 1.0, buffers=bufs)
+
+    for _ in range(3):
+        block()
+    sync()
+    stepper = Stepper(block, 1, dev, no_graph)
+    times, clocks, _ = timed_repetitions(stepper, 4, sync, 1, dev, local, min_reps=10)
+    block_s = median(times) / 4
+
+    def layer(xin, w, M, N, K):
+        ws = quest.alloc_workspace(M, N, K, BITS, BITS, dev)
+        out = quest.quest_linear_fwd(xin, w, BITS, 128, 1.0, workspace=ws)
+        st = Stepper(lambda i: quest.quest_linear_fwd(xin, w, BITS, 128, 1.0, y=out["y"], saved=out, workspace=ws), 1, dev, no_graph)
+        sm = stage_times(quest, st, 1, reps=20)
+        g_tops = 2.0 * M * N * K / (sm["gemm"] * 1e-3) / 1e12
+        q_gbs = (quantizer_bytes(M, K, BITS) + quantizer_bytes(N, K, BITS)) / (sm["quant_x"] * 1e-3) / 1e9
+        return {"shape": f"{M}x{N}x{K}", "gemm_ms": sm["gemm"], "gemm_tops": g_tops,
+                "gemm_frac": {k: g_tops / v for k, v in int8_peaks.items() if v},
+                "quant_ms": sm["quant_x"], "quant_gbs": q_gbs, "quant_frac_hbm": q_gbs / peaks["hbm_gbs"],
+                "quantizes": f"x[{M}x{K}] and w[{N}x{K}] in one launch"}
+
+    gate = layer(x, wg, T, I, H)
+    h = bufs["h"]
+    down = layer(h, wd, T, H, I)
+    # the quantizer alone on h[8192 x 5504] (activations only, as in the cached-weight pipeline)
+    cb = quest.container_bits(BITS)
+    qc = torch.empty((T, I * cb // 8), dtype=torch.uint8, device=dev)
+    qs = torch.empty(T, dtype=torch.float32, device=dev)
+    qm = torch.empty((T, I // 8), dtype=torch.uint8, device=dev)
+    qst = Stepper(lambda i: quest.quest_quantize(h, BITS, 128, 1.0, codes=qc, scales=qs, mask=qm), 1, dev, no_graph)
+    qt, _, _ = timed_repetitions(qst, 4, sync, 1, dev, local, min_reps=10)
+    qh_s = median(qt) / 4
+    qh_gbs = quantizer_bytes(T, I, BITS) / qh_s / 1e9
+    flops = 2.0 * T * (2 * I * H + H * I)
+    return {"workload": "config 4: Llama MLP block fwd, X[8192x2048], gate/up W[5504x2048], down W[2048x5504], bf16, b=4, g=128",
+            "block_us": 1e6 * block_s, "block_tokens_per_s": T / block_s, "block_tops": flops / block_s / 1e12,
+            "block_frac": {k: flops / block_s / 1e12 / v for k, v in int8_peaks.items() if v},
+            "block_launches": bufs["launches"], "block_call": "quest_mlp_fwd, replayed from one CUDA graph",
+            "repetitions": len(times),
+            "gate_or_up_layer": gate, "down_layer": down,
+            "quantizer_on_h": {"ms": 1e3 * qh_s, "gbs": qh_gbs, "frac_hbm": qh_gbs / peaks["hbm_gbs"],
+                               "note": "quest_quantize alone (no GEMM operand written), graph replay, no event nodes"},
+            "clocks": clocks.summary(), "stage_ms_includes": BRACKETED}
+
+
 # ------------------------------------------------------------------------------------ GPU arm
 
 def run_gpu(args, rank: int, world: int, local: int):
@@ -266,71 +545,29 @@ def run_gpu(args, rank: int, world: int, local: int):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # The steps are replayed from a CUDA graph holding one pass over the ring (n_sets steps), so
-    # that the host's launch rate does not bound a step of a few tens of microseconds; the
-    # remainder K mod n_sets is launched directly.  --no-graph launches every step directly.
-    side = torch.cuda.Stream(device=dev)
-
-    def run_steps(fn, k, graph):
-        if graph is None:
-            for i in range(k):
-                fn(i)
-            return
-        for _ in range(k // n_sets):
-            graph.replay()
-        for i in range(k % n_sets):
-            fn(i)
-
-    def capture(fn):
-        if args.no_graph:
-            return None
-        g_ = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            for i in range(n_sets):
-                fn(i)
-            side.synchronize()
-            with torch.cuda.graph(g_, stream=side):
-                for i in range(n_sets):
-                    fn(i)
-        torch.cuda.synchronize()
-        return g_
-
-    # ---- device-resident timing -------------------------------------------------------
+    # ---- device-resident timing: the block of K steps, repeated ------------------------------
     for i in range(max(args.warmup, 3)):
         step(i)
     barrier()
-    graph = capture(step)
-    run_steps(step, n_sets, graph)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        e0.record()
-        run_steps(step, args.steps, graph)
-        e1.record()
-        torch.cuda.synchronize()
-    elapsed_s = e0.elapsed_time(e1) * 1e-3
-    barrier()
+    stepper = Stepper(step, n_sets, dev, args.no_graph)
+    times, clocks, mhz = timed_repetitions(stepper, args.steps, barrier, world, dev, local)
     status = quest.quest_device_status()
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
-    max_elapsed = max_over_ranks(elapsed_s, world, dev)
+    max_elapsed = median(times)
     value = aggregate_tokens_per_s(M, args.steps, world, max_elapsed)
 
     # ---- two labelled variants of the same step (not the headline): (1) weight codes cached from an
     # earlier call, the inference pipeline of Section 5: only X is quantized, W's tensor-core operand is kept in the
     # workspace from the earlier call (w_is_cached = 2);
     # (2) L2-warm: every step on the same buffer set, so inputs and outputs stay in the 126 MB L2.
-    def time_variant(fn, k):
-        gv = capture(fn)
-        run_steps(fn, n_sets, gv)
-        torch.cuda.synchronize()
-        v0, v1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        v0.record()
-        run_steps(fn, k, gv)
-        v1.record()
-        torch.cuda.synchronize()
-        t = max_over_ranks(v0.elapsed_time(v1) * 1e-3, world, dev)
-        return {"value": aggregate_tokens_per_s(M, k, world, t), "unit": UNIT, "ms_per_step": 1e3 * t / k, "steps": k}
+    def time_variant(fn):
+        k = args.steps
+        st = Stepper(fn, n_sets, dev, args.no_graph)
+        t, _, _ = timed_repetitions(st, k, barrier, world, dev, local, min_reps=5)
+        m = median(t)
+        return {"value": aggregate_tokens_per_s(M, k, world, m), "unit": UNIT, "ms_per_step": 1e3 * m / k, "steps": k,
+                "repetitions": len(t)}
 
     def step_cached(i):
         s = ring[i % n_sets]
@@ -342,28 +579,11 @@ def run_gpu(args, rank: int, world: int, local: int):
         s = ring[0]
         quest.quest_linear_fwd(s["x"], s["w"], BITS, g, 1.0, y=s["y"], saved=s["saved"], workspace=s["ws"])
 
-    v_steps = min(args.steps, 300)
-    variants = {"cached_weight_codes": time_variant(step_cached, v_steps), "l2_warm": time_variant(step_warm, v_steps)}
+    variants = {"cached_weight_codes": time_variant(step_cached), "l2_warm": time_variant(step_warm)}
     barrier()
 
-    # ---- per-kernel durations: the same steps with every stage bracketed by CUDA events on the
-    # launching stream.  With a graph the event records are graph nodes, so the host's launch
-    # rate does not sit between an event and its kernel; each replay yields the stage times of
-    # the graph's last step.
-    quest.quest_stage_timing(True)
-    quest.quest_stage_times(reset=2)
-    staged = capture(step)
-    prof_reps = 50
-    for r in range(prof_reps):
-        if staged is None:
-            step(r)
-        else:
-            staged.replay()
-        quest.quest_stage_times()
-    stage = quest.quest_stage_times(reset=2)
-    quest.quest_stage_timing(False)
-    del staged
-    stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+    stage_ms = stage_times(quest, stepper, n_sets)
+    overhead_ms = bracket_overhead_ms(dev)
 
     # ---- end to end: pinned host inputs in, result out, every step ---------------------
     # Each step copies x and w from pinned host memory, runs the C ABI call and copies y back to
@@ -376,7 +596,7 @@ def run_gpu(args, rank: int, world: int, local: int):
     e2e_sets = (n_sets // n_lanes) * n_lanes if n_sets >= n_lanes else n_lanes
     while len(ring) < e2e_sets:
         ring.append(make_set())
-    e2e_steps = min(args.steps, 200)
+    e2e_steps = min(max(args.steps, 60), 200)
 
     def e2e_step(i):
         s = ring[i % e2e_sets]
@@ -404,11 +624,13 @@ def run_gpu(args, rank: int, world: int, local: int):
         return start.elapsed_time(stop) * 1e-3
 
     e2e_run(2 * e2e_sets)
-    barrier()
-    e2e_local = e2e_run(e2e_steps)
-    y_host = y_hosts[0]
-    e2e_elapsed = max_over_ranks(e2e_local, world, dev)
+    e2e_times = []
+    for _ in range(3):
+        barrier()
+        e2e_times.append(e2e_run(e2e_steps))
+    e2e_elapsed = median(max_over_ranks(e2e_times, world, dev))
     e2e_value = aggregate_tokens_per_s(M, e2e_steps, world, e2e_elapsed)
+    y_host = y_hosts[0]
     h2d = x_host.numel() * 2 + w_host.numel() * 2
     d2h = y_host.numel() * 2
 
@@ -419,10 +641,15 @@ def run_gpu(args, rank: int, world: int, local: int):
         return
 
     peaks = load_peaks()
+    counters = load_ncu_counters()
     src = "of measured" if peaks["_source"] == "measured" else "of fallback"
     # one- and two-bit codes run on the FP4 tensor-core path (nominal rate twice that of int8)
     fp4_path = BITS <= 2
-    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16 * (2.0 if fp4_path else 1.0)
+    rate = 2.0 if fp4_path else 1.0
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16 * rate
+    lib_same = library_int8_tops(dev, M, N, K)
+    lib_8192 = library_int8_tops(dev, 8192, 8192, 8192, iters=10)
+    int8_peaks = {"of_2x_bf16_burst": int8_peak, "of_library_int8_gemm_8192": lib_8192 * rate if lib_8192 else None}
     gemm_ms = stage_ms["gemm"]
     gemm_tops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12 if gemm_ms else None
     qx_bytes, qw_bytes = quantizer_bytes(M, K, BITS), quantizer_bytes(N, K, BITS)
@@ -430,23 +657,17 @@ def run_gpu(args, rank: int, world: int, local: int):
     q_ms = stage_ms["quant_x"]
     q_bytes = qx_bytes + qw_bytes
     q_gbs = q_bytes / (q_ms * 1e-3) / 1e9 if q_ms else None
+    gemm_c = counters.get("gemm_config2") if BITS == 4 else None
+    quant_c = counters.get("quantizer_config2") if (BITS == 4 and g == 128) else None
+    mhz_med = clocks.summary()["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)
+    ipe = quant_c.get("thread_instructions_per_element") if quant_c else None
 
-    # int8 library GEMM on the same shape, as a cross-check of the tensor-pipe denominator
-    lib_tops = None
-    try:
-        a8 = torch.randint(-8, 8, (M, K), dtype=torch.int8, device=dev)
-        b8 = torch.randint(-8, 8, (K, N), dtype=torch.int8, device=dev)
-        for _ in range(3):
-            torch._int_mm(a8, b8)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(20):
-            torch._int_mm(a8, b8)
-        e1.record()
-        torch.cuda.synchronize()
-        lib_tops = 2.0 * M * N * K * 20 / (e0.elapsed_time(e1) * 1e-3) / 1e12
-    except Exception:
-        lib_tops = None
+    config4 = None
+    if not args.no_config4 and BITS == 4 and world == 1:
+        try:
+            config4 = run_config4(quest, dev, peaks, int8_peaks, args.no_graph)
+        except Exception as e:                                   # the headline must not depend on it
+            config4 = {"error": f"{type(e).__name__}: {e}"}
 
     sample = args.ref_tokens if args.ref_tokens > 0 else TOKENS
     o_dt, o_threads = time_oracle(sample, g)
@@ -457,10 +678,13 @@ def run_gpu(args, rank: int, world: int, local: int):
         "data": "synthetic",
         "config": dict(workload_config(g), parallelism=f"replicas x{world}",
                        l2="ring of %d buffer sets (%.0f MB) larger than L2; no flush" % (n_sets, n_sets * set_bytes / 1e6)),
+        "timing": "median over repetitions of the block of `steps` steps; each repetition bracketed by barrier + "
+                  "synchronize, CUDA events on the launching stream, max over ranks",
+        "repetitions": spread(times, args.steps, mhz),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "launch": f"direct, {n_lanes} streams in rotation"},
-        "gpu_launches": 2 * args.steps,     # per step: one quantizer launch (x and w together), one GEMM launch
-        "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
+                "steps": e2e_steps, "repetitions": len(e2e_times), "launch": f"direct, {n_lanes} streams in rotation"},
+        "gpu_launches": 2 * args.steps,     # per timed block; per step: one quantizer launch (x and w together), one GEMM launch
+        "launch": stepper.launch_mode(args.steps),
         "clocks": clocks.summary(),
         "roofline": {"bound": "tensor",
                      "kernel": "gemm_i8_kernel<mode 5> (tcgen05 kind::mxf4 on E2M1 operands)" if fp4_path
@@ -468,24 +692,29 @@ def run_gpu(args, rank: int, world: int, local: int):
                      "achieved": gemm_tops,
                      "peak": int8_peak, "unit": "TOP/s", "frac": (gemm_tops / int8_peak) if gemm_tops else None,
                      "peak_basis": f"{4 if fp4_path else 2} x bf16 burst {src} ({peaks['bf16_tflops']} TFLOP/s)",
-                     "traffic": GEMM_DRAM_TRAFFIC_BYTES if BITS == 4 else None, "ms": gemm_ms,
-                     "library_int8_gemm_tops_same_shape": lib_tops},
+                     "frac_of_library_int8_gemm_8192": (gemm_tops / (lib_8192 * rate)) if (gemm_tops and lib_8192) else None,
+                     "library_int8_gemm_8192_tops": lib_8192,
+                     "library_int8_gemm_tops_same_shape": lib_same,
+                     "traffic": gemm_c.get("dram_bytes") if gemm_c else None,
+                     "traffic_source": gemm_c.get("source") if gemm_c else None,
+                     "ms": gemm_ms, "ms_includes": BRACKETED},
         "roofline_quantizer": {"bound": "hbm", "kernel": "quantizer, x and w rows in one launch", "achieved": q_gbs,
                                "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": (q_gbs / peaks["hbm_gbs"]) if q_gbs else None, "peak_basis": src,
-                               "traffic": QUANT_DRAM_TRAFFIC_BYTES if BITS == 4 else None, "ms": q_ms,
+                               "traffic": quant_c.get("dram_bytes") if quant_c else None,
+                               "traffic_source": quant_c.get("source") if quant_c else None,
+                               "ms": q_ms, "ms_includes": BRACKETED,
                                "algorithmic_bytes": q_bytes,
-                               # the kernel is bound by instruction issue, not HBM: the same launch against the
-                               # issue rate 148 SMs x 4 schedulers x 32 lanes x SM clock
-                               "alu": (lambda mhz: {"bound": "alu", "unit": "T thread-instr/s",
-                                                    "achieved": QUANT_INSTR_PER_ELEMENT * (M + N) * K / (q_ms * 1e-3) / 1e12,
-                                                    "peak": 148 * 4 * 32 * mhz * 1e6 / 1e12,
-                                                    "frac": QUANT_INSTR_PER_ELEMENT * (M + N) * K / (q_ms * 1e-3)
-                                                            / (148 * 4 * 32 * mhz * 1e6),
-                                                    "instr_per_element": QUANT_INSTR_PER_ELEMENT})(
-                                   clocks.summary()["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)) if (q_ms and BITS == 4) else None},
+                               # the same launch against the issue rate 148 SMs x 4 schedulers x 32 lanes x SM clock
+                               "alu": {"bound": "alu", "unit": "T thread-instr/s",
+                                       "achieved": ipe * (M + N) * K / (q_ms * 1e-3) / 1e12,
+                                       "peak": 148 * 4 * 32 * mhz_med * 1e6 / 1e12,
+                                       "frac": ipe * (M + N) * K / (q_ms * 1e-3) / (148 * 4 * 32 * mhz_med * 1e6),
+                                       "instr_per_element": ipe} if (q_ms and ipe) else None},
         "stage_ms": stage_ms,
-        "variants": variants,
+        "stage_ms_includes": BRACKETED,
+        "event_bracket_overhead_ms": overhead_ms,
+        "variants": dict(variants, config4=config4),
         "cpu_baseline": {"value": sample / o_dt, "unit": UNIT, "cores": o_threads, "kind": "oracle",
                          "sample": f"{sample} of {TOKENS} token rows against the full W, one pass"},
     }
@@ -530,59 +759,17 @@ def run_backward(args, rank: int, world: int, local: int):
         s = ring[i % n_sets]
         quest.quest_linear_bwd(s["dy"], fwd, BITS, g, K, dx=s["dx"], dw=s["dw"], workspace=s["ws"])
 
-    def capture():
-        if args.no_graph:
-            return None
-        side = torch.cuda.Stream(device=dev)
-        g_ = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            for i in range(n_sets):
-                step(i)
-            side.synchronize()
-            with torch.cuda.graph(g_, stream=side):
-                for i in range(n_sets):
-                    step(i)
-        torch.cuda.synchronize()
-        return g_
-
-    def run_steps(k, graph):
-        if graph is None:
-            for i in range(k):
-                step(i)
-            return
-        for _ in range(k // n_sets):
-            graph.replay()
-        for i in range(k % n_sets):
-            step(i)
-
+    sync = lambda: torch.cuda.synchronize()
     for i in range(max(args.warmup, 3)):
         step(i)
-    torch.cuda.synchronize()
-    graph = capture()
-    run_steps(n_sets, graph)
-    torch.cuda.synchronize()
+    sync()
+    stepper = Stepper(step, n_sets, dev, args.no_graph)
     steps = min(args.steps, 300)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        e0.record()
-        run_steps(steps, graph)
-        e1.record()
-        torch.cuda.synchronize()
-    elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3, world, dev)
+    times, clocks, mhz = timed_repetitions(stepper, steps, sync, world, dev, local)
+    elapsed = median(times)
     if quest.quest_device_status() != 0:
         raise RuntimeError("device status after the timed region")
-    quest.quest_stage_timing(True)
-    quest.quest_stage_times(reset=2)
-    staged = capture()
-    for r in range(30):
-        if staged is None:
-            step(r)
-        else:
-            staged.replay()
-        quest.quest_stage_times()
-    stage = quest.quest_stage_times(reset=2)
-    quest.quest_stage_timing(False)
-    stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+    stage_ms = stage_times(quest, stepper, n_sets, reps=30)
     if rank != 0:
         return
     peaks = load_peaks()
@@ -603,13 +790,14 @@ def run_backward(args, rank: int, world: int, local: int):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": dict(workload_config(g), workload="config 2, Algorithm 2 (backward): dy[4096x2048] bf16 -> dx, dw bf16",
                        l2="ring of %d buffer sets (%.0f MB) larger than L2" % (n_sets, n_sets * set_bytes / 1e6)),
-        "gpu_launches": 3 * steps, "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
+        "repetitions": spread(times, steps, mhz),
+        "gpu_launches": 3 * steps, "launch": stepper.launch_mode(steps),
         "clocks": clocks.summary(),
         "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel<mode 3> (tcgen05 kind::f16 bf16, MN-major operands, fused mask + inverse Hadamard)",
                      "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": (tflops / peaks["bf16_tflops"]) if tflops else None,
                      "peak_basis": "bf16 burst " + ("of measured" if peaks["_source"] == "measured" else "of fallback"),
-                     "traffic": None, "ms": gemm_ms},
+                     "traffic": None, "ms": gemm_ms, "ms_includes": BRACKETED},
         "stage_ms": {"prepare": stage_ms["unpack"], "gemm_last": gemm_ms},
         "cpu_baseline": {"value": M * frac / o_dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
                          "sample": "64 rows of dL/dx and 64 rows of dL/dw (binary64 numpy), scaled by their share of the flops"},
@@ -652,59 +840,17 @@ def run_weight_only(args, rank: int, world: int, local: int):
         s = ring[i % n_sets]
         quest.quest_linear_fwd_weight_only(s["x"], s["w"], BITS, g, 1.0, out=s["out"], workspace=s["ws"])
 
-    def capture():
-        if args.no_graph:
-            return None
-        side = torch.cuda.Stream(device=dev)
-        g_ = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            for i in range(n_sets):
-                step(i)
-            side.synchronize()
-            with torch.cuda.graph(g_, stream=side):
-                for i in range(n_sets):
-                    step(i)
-        torch.cuda.synchronize()
-        return g_
-
-    def run_steps(k, graph):
-        if graph is None:
-            for i in range(k):
-                step(i)
-            return
-        for _ in range(k // n_sets):
-            graph.replay()
-        for i in range(k % n_sets):
-            step(i)
-
+    sync = lambda: torch.cuda.synchronize()
     for i in range(max(args.warmup, 3)):
         step(i)
-    torch.cuda.synchronize()
-    graph = capture()
-    run_steps(n_sets, graph)
-    torch.cuda.synchronize()
+    sync()
+    stepper = Stepper(step, n_sets, dev, args.no_graph)
     steps = min(args.steps, 500)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        e0.record()
-        run_steps(steps, graph)
-        e1.record()
-        torch.cuda.synchronize()
-    elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3, world, dev)
+    times, clocks, mhz = timed_repetitions(stepper, steps, sync, world, dev, local)
+    elapsed = median(times)
     if quest.quest_device_status() != 0:
         raise RuntimeError("device status after the timed region")
-    quest.quest_stage_timing(True)
-    quest.quest_stage_times(reset=2)
-    staged = capture()
-    for r in range(30):
-        if staged is None:
-            step(r)
-        else:
-            staged.replay()
-        quest.quest_stage_times()
-    stage = quest.quest_stage_times(reset=2)
-    quest.quest_stage_timing(False)
-    stage_ms = {k: (tot / cnt if cnt else None) for k, (tot, cnt) in stage.items()}
+    stage_ms = stage_times(quest, stepper, n_sets, reps=30)
     if rank != 0:
         return
     peaks = load_peaks()
@@ -721,13 +867,14 @@ def run_weight_only(args, rank: int, world: int, local: int):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": dict(workload_config(g), workload="config 2, weight-only: X[4096x2048] bf16 x W4[2048x2048] -> y bf16",
                        l2="ring of %d buffer sets (%.0f MB) larger than L2" % (n_sets, n_sets * set_bytes / 1e6)),
-        "gpu_launches": 2 * steps, "launch": "direct" if args.no_graph else f"CUDA graph of {n_sets} steps replayed",
+        "repetitions": spread(times, steps, mhz),
+        "gpu_launches": 2 * steps, "launch": stepper.launch_mode(steps),
         "clocks": clocks.summary(),
         "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel<mode 4> (tcgen05 kind::f16 bf16, column-scale epilogue)",
                      "achieved": tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                      "frac": (tflops / peaks["bf16_tflops"]) if tflops else None,
                      "peak_basis": "bf16 burst " + ("of measured" if peaks["_source"] == "measured" else "of fallback"),
-                     "traffic": None, "ms": gemm_ms},
+                     "traffic": None, "ms": gemm_ms, "ms_includes": BRACKETED},
         "stage_ms": {"rotate_and_quantize": stage_ms["quant_w"], "gemm": gemm_ms},
         "cpu_baseline": {"value": sample / o_dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
                          "sample": "%d of %d token rows against the full W (weights quantized in full)" % (sample, M)},
@@ -738,11 +885,12 @@ def run_weight_only(args, rank: int, world: int, local: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=250)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="quest", choices=["quest", "reference"])
     ap.add_argument("--had-block", type=int, default=128)
     ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-config4", action="store_true", help="skip the config-4 MLP block variant")
     ap.add_argument("--pass", dest="which", default="forward", choices=["forward", "backward", "weight_only"],
                     help="forward: Algorithm 1, the headline metric (default); backward: Algorithm 2 on the same layer; "
                          "weight_only: the W4A16 forward of Section 4.5 on the same layer")

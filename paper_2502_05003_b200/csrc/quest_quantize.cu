@@ -821,6 +821,304 @@ quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
     rotate_project_store<CB, 32, true, true, GRID, false, RS>(v, a, tn, active, row, tr, r_local, xsm, 32);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Block kernel: bfloat16 rows stored densely, had_block = 128, codes + scales + mask requested,
+// trust_factor >= 1.  ONE THREAD OWNS ONE WHOLE ROTATION BLOCK of 128 elements, so no butterfly
+// stage crosses a thread (no shuffles at all in the rotation) and the per-thread costs (index
+// arithmetic, the row's RMS and reciprocal, stores) are spread over 128 elements instead of 32.
+// A warp's 32 blocks are 8 KB of consecutive memory.  They are fetched with coalesced 16-byte loads
+// (a warp instruction reads 512 consecutive bytes) and redistributed through a swizzled
+// shared-memory tile so that every thread ends up with its own 256 bytes; packed codes and the
+// int8 GEMM operand travel the same way in the other direction.  The trust mask needs no detour:
+// a thread's 16 bytes of mask follow its neighbour's.
+// The sum of squares of a block is a complete subtree of the row's canonical pairwise tree, so
+// the threads of a row combine their block sums in the same order as every other kernel: by
+// xor-shuffles when a row has a power-of-two number of blocks of at most 32, through shared memory
+// otherwise.
+// ---------------------------------------------------------------------------------------------
+constexpr int BLK_TILE_BYTES = 8192;             // per warp: 32 blocks x 256 bytes of bfloat16
+
+// Levels, mask bits and packed code words of 32 consecutive rotated elements (16 float2 pairs), for
+// trust_factor >= 1: an element inside the grid is within half a step of its level, so only clipped
+// elements can be masked, and for those the level is the clamp bound itself.
+template <int CB, int GRID>
+__device__ __forceinline__ void project32_trusting(const float2 *v, float inv, const QuantConsts &qc, uint32_t (&w)[CB],
+                                                   uint32_t &mask_word) {
+    const float2 neg1 = make_float2(-1.0f, -1.0f);
+    const float hh = qc.h;
+    uint32_t mbits = 0;
+    if constexpr (GRID == GRID_FP4) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float t[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                t[2 * j] = __fmul_rn(v[q * 4 + j].x, inv);
+                t[2 * j + 1] = __fmul_rn(v[q * 4 + j].y, inv);
+            }
+            w[q] = cvt_e2m1x8(t);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                mbits |= (__fsub_rn(fabsf(t[j]), 6.0f) <= hh ? 1u : 0u) << (q * 8 + j);
+        }
+        mask_word = mbits;
+    } else {
+        const float2 inv2 = make_float2(inv, inv), c02 = make_float2(qc.c0, qc.c0);
+        const float2 magic2 = make_float2(QUEST_MAGIC_RNE, QUEST_MAGIC_RNE);
+        const float top = qc.top;
+        uint32_t kb[32];                                        // MAGIC_BITS + level
+        uint32_t mhi = 0;                                       // elements 16..31 (two independent shift chains)
+#pragma unroll
+        for (int i = 7; i >= 0; --i) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int p = i + 8 * half;
+                const float2 t = __ffma2_rn(v[p], inv2, c02);
+                float2 tc;
+                tc.x = fminf(fmaxf(t.x, 0.0f), top);
+                tc.y = fminf(fmaxf(t.y, 0.0f), top);
+                const float2 km = __fadd2_rn(tc, magic2);
+                const float2 d = __ffma2_rn(tc, neg1, t);       // t - clamp(t)
+                const float dy = __fsub_rn(hh, fabsf(d.y));     // >= +0  <=>  trusted
+                const float dx = __fsub_rn(hh, fabsf(d.x));
+                uint32_t &m = half ? mhi : mbits;
+                m = __funnelshift_l(__float_as_uint(dy), m, 1); // sign bit: 1 = masked
+                m = __funnelshift_l(__float_as_uint(dx), m, 1);
+                kb[2 * p] = __float_as_uint(km.x);
+                kb[2 * p + 1] = __float_as_uint(km.y);
+            }
+        }
+        mask_word = ~__byte_perm(mbits, mhi, 0x5410);           // low halves: elements 0..15 | 16..31
+        constexpr int PER = 32 / CB;
+        uint32_t magic_sum = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) magic_sum += QUEST_MAGIC_BITS << (CB * j);
+#pragma unroll
+        for (int q = 0; q < CB; ++q) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int j = PER - 1; j >= 0; --j) acc = (acc << CB) + kb[q * PER + j];
+            w[q] = acc - magic_sum;
+        }
+    }
+}
+
+// Swizzled position of 16-byte chunk `j` in row `r` of a tile whose rows hold NC chunks (NC = 4, 8 or
+// 16): both the row-wise accesses of one thread per row and the chunk-wise accesses of consecutive
+// lanes fall into distinct bank groups.
+template <int NC>
+__device__ __forceinline__ int swz(int r, int j) {
+    if constexpr (NC == 4) return j ^ ((r >> 1) & 3);
+    else return j ^ (r & 7);
+}
+
+// Copies a warp tile of 32 rows x NC chunks from shared memory to consecutive global memory.
+template <int NC>
+__device__ __forceinline__ void tile_to_global(const uint8_t *tile, uint8_t *dst, int lane, int live_rows) {
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+        const int c = i * 32 + lane;
+        const int r = c / NC, j = c % NC;
+        if (r < live_rows)
+            *reinterpret_cast<uint4 *>(dst + (size_t)c * 16) =
+                *reinterpret_cast<const uint4 *>(tile + r * (NC * 16) + swz<NC>(r, j) * 16);
+    }
+}
+
+template <int CB, int GRID>
+__global__ void __launch_bounds__(128, 3)
+quantize_block128_kernel(const __grid_constant__ QuantArgs a) {
+    extern __shared__ __align__(16) uint8_t smem_raw[];   // [warps][8 KB] tiles, then [threads] + [rows] floats
+    pdl_launch_dependents();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
+    const QuantTensor &tn = a.t[which];
+    const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
+    const int cols = a.cols;
+    const int T = cols >> 7;                                   // blocks (= threads) per row
+    const long long row0 = (long long)blk * a.R;
+    const long long rows_left = tn.rows - row0;
+    const int rows_here = rows_left < a.R ? (int)rows_left : a.R;
+    const int nslots = rows_here * T;                          // live (row, block) slots of this CTA
+    const bool active = tid < nslots;
+    uint8_t *tile = smem_raw + warp * BLK_TILE_BYTES;
+    float *part = reinterpret_cast<float *>(smem_raw + nwarps * BLK_TILE_BYTES);
+    float *rowss = part + blockDim.x;
+    const int wslot0 = warp * 32;
+    const int wlive = nslots - wslot0 < 32 ? nslots - wslot0 : 32;     // live slots of this warp (may be <= 0)
+    const size_t first_elem = (size_t)row0 * cols + (size_t)wslot0 * 128;   // dense rows: slots are consecutive blocks
+
+    // ---- fetch: coalesced 16-byte loads, then every thread takes its own block from the tile -----
+    float2 v[64];
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(tn.x) + first_elem);
+        uint4 raw[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int c = q * 32 + lane;
+            raw[q] = (c >> 4) < wlive ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int c = q * 32 + lane;
+            const int r = c >> 4, j = c & 15;
+            *reinterpret_cast<uint4 *>(tile + r * 256 + swz<16>(r, j) * 16) = raw[q];
+        }
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(tile + lane * 256 + swz<16>(lane, q) * 16);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                v[q * 4 + j] = make_float2(__uint_as_float(ww[j] << 16), __uint_as_float(ww[j] & 0xFFFF0000u));
+        }
+        __syncwarp();                                          // the tile is reused for the outputs
+    }
+
+    // ---- rotation: strides 64 .. 2 on pairs, then stride 1 inside the pairs ---------------------
+    {
+        const float2 neg1 = make_float2(-1.0f, -1.0f);
+#pragma unroll
+        for (int s2 = 32; s2 >= 1; s2 >>= 1) {
+#pragma unroll
+            for (int i = 0; i < 64; ++i)
+                if ((i & s2) == 0) {
+                    const float2 p = v[i], q = v[i + s2];
+                    v[i] = __fadd2_rn(p, q);
+                    v[i + s2] = __ffma2_rn(q, neg1, p);        // p - q
+                }
+        }
+#pragma unroll
+        for (int i = 0; i < 64; ++i) {
+            const float p = v[i].x, q = v[i].y;
+            v[i] = make_float2(__fadd_rn(p, q), __fsub_rn(p, q));
+        }
+    }
+
+    // ---- sum of squares of the block: the canonical pairwise tree, two half-blocks per packed add ---
+    float ss;
+    {
+        float2 p[32];                                          // (sum over elements 2i, 2i+1; the same 64 elements later)
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const float2 lo = __fmul2_rn(v[i], v[i]), hi = __fmul2_rn(v[i + 32], v[i + 32]);
+            p[i] = make_float2(__fadd_rn(lo.x, lo.y), __fadd_rn(hi.x, hi.y));
+        }
+#pragma unroll
+        for (int n = 16; n >= 1; n >>= 1)
+#pragma unroll
+            for (int i = 0; i < n; ++i) p[i] = __fadd2_rn(p[2 * i], p[2 * i + 1]);
+        ss = __fadd_rn(p[0].x, p[0].y);
+    }
+    // ---- the row's sum: block sums combined pairwise over the zero-padded row -------------------
+    int my_row, my_t;
+    if ((T & (T - 1)) == 0 && T <= 32) {                       // uniform over the launch
+        for (int m = 1; m < T; m <<= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, m));
+        const int sh = 31 - __clz(T);
+        my_row = tid >> sh;
+        my_t = tid & (T - 1);
+    } else {
+        part[tid] = ss;                                        // slots past the end hold zeros
+        __syncthreads();
+        for (int r = warp; r < rows_here; r += nwarps) {
+            float acc[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = lane + 32 * k;
+                acc[k] = i < T ? part[r * T + i] : 0.0f;
+#pragma unroll
+                for (int m = 1; m < 32; m <<= 1) acc[k] = __fadd_rn(acc[k], __shfl_xor_sync(0xffffffffu, acc[k], m));
+            }
+            const float tot = __fadd_rn(__fadd_rn(acc[0], acc[1]), __fadd_rn(acc[2], acc[3]));
+            if (lane == 0) rowss[r] = tot;
+        }
+        __syncthreads();
+        my_row = active ? tid / T : 0;
+        my_t = tid - my_row * T;
+        ss = rowss[my_row < rows_here ? my_row : 0];
+    }
+    const float rms = __fsqrt_rn(__fdiv_rn(ss, (float)cols));
+    const float inv = (rms > 0.0f) ? __fdiv_rn(a.qc.A, rms) : 0.0f;
+    const long long row = row0 + my_row;
+    if (active && my_t == 0) tn.scales[row] = __fmul_rn(rms, a.qc.B);
+
+    // ---- project 4 x 32 elements; codes and operand bytes go to the tile, mask words stay here ---
+    constexpr int CODE_NC = CB >= 4 ? CB : 4;                  // 16-byte chunks per thread's row of codes (CB = 4, 8)
+    constexpr bool E2M1_OP = CB <= 2;
+    uint8_t *code_tile = tile;                                 // [32][CODE_NC x 16] (CB >= 4 only)
+    uint8_t *op_tile = tile + 4096;                            // [32][OP_NC x 16]
+    const bool want_op = GRID == GRID_UNIFORM && tn.op8 != nullptr;
+    uint32_t mw[4];
+    uint32_t small_codes[CB <= 2 ? 4 * CB : 1];                // one- and two-bit codes: 16 or 32 bytes per thread
+#pragma unroll
+    for (int g32 = 0; g32 < 4; ++g32) {
+        uint32_t w[CB];
+        project32_trusting<CB, GRID>(&v[g32 * 16], inv, a.qc, w, mw[g32]);
+        if constexpr (CB == 4) {
+            *reinterpret_cast<uint4 *>(code_tile + lane * 64 + swz<4>(lane, g32) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        } else if constexpr (CB == 8) {
+            *reinterpret_cast<uint4 *>(code_tile + lane * 128 + swz<8>(lane, 2 * g32) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(code_tile + lane * 128 + swz<8>(lane, 2 * g32 + 1) * 16) = make_uint4(w[4], w[5], w[6], w[7]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < CB; ++q) small_codes[g32 * CB + q] = w[q];
+        }
+        if constexpr (GRID == GRID_UNIFORM) {
+            if (want_op) {                                     // uniform over the CTA
+                if constexpr (E2M1_OP) {
+                    uint32_t o[4];
+                    e2m1_operand_from_code_words<CB>(w, o);
+                    *reinterpret_cast<uint4 *>(op_tile + lane * 64 + swz<4>(lane, g32) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+                } else {
+                    uint32_t o[8];
+                    operand_from_code_words<CB>(w, a.bits, o);
+                    *reinterpret_cast<uint4 *>(op_tile + lane * 128 + swz<8>(lane, 2 * g32) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4 *>(op_tile + lane * 128 + swz<8>(lane, 2 * g32 + 1) * 16) = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+            }
+        }
+    }
+    // ---- stores ------------------------------------------------------------------------------------
+    if (active)                                                // 16 bytes of mask per block, consecutive across lanes
+        *reinterpret_cast<uint4 *>(tn.mask + (first_elem >> 3) + (size_t)lane * 16) = make_uint4(mw[0], mw[1], mw[2], mw[3]);
+    if constexpr (CB == 1) {
+        if (active) *reinterpret_cast<uint4 *>(tn.codes + (first_elem >> 3) + (size_t)lane * 16) =
+                        make_uint4(small_codes[0], small_codes[1], small_codes[2], small_codes[3]);
+    } else if constexpr (CB == 2) {
+        if (active) {
+            uint4 *dst = reinterpret_cast<uint4 *>(tn.codes + (first_elem >> 2) + (size_t)lane * 32);
+            dst[0] = make_uint4(small_codes[0], small_codes[1], small_codes[2], small_codes[3]);
+            dst[1] = make_uint4(small_codes[4], small_codes[5], small_codes[6], small_codes[7]);
+        }
+    }
+    __syncwarp();
+    if (wlive > 0) {
+        if constexpr (CB >= 4) tile_to_global<CODE_NC>(code_tile, tn.codes + first_elem * CB / 8, lane, wlive);
+        if constexpr (GRID == GRID_UNIFORM) {
+            if (want_op) {
+                if constexpr (E2M1_OP) tile_to_global<4>(op_tile, reinterpret_cast<uint8_t *>(tn.op8) + (first_elem >> 1), lane, wlive);
+                else tile_to_global<8>(op_tile, reinterpret_cast<uint8_t *>(tn.op8) + first_elem, lane, wlive);
+            }
+        }
+    }
+}
+
+template <int GRID>
+static cudaError_t launch_block128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
+    if constexpr (GRID == GRID_FP4) {
+        return launch_pdl(quantize_block128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
+    } else {
+        switch (cb) {
+            case 1: return launch_pdl(quantize_block128_kernel<1, GRID>, grid, dim3(threads), smem, st, 1, a);
+            case 2: return launch_pdl(quantize_block128_kernel<2, GRID>, grid, dim3(threads), smem, st, 1, a);
+            case 4: return launch_pdl(quantize_block128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
+            default: return launch_pdl(quantize_block128_kernel<8, GRID>, grid, dim3(threads), smem, st, 1, a);
+        }
+    }
+}
+
 template <int GRID>
 static cudaError_t launch_direct128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                     bool rowsums = false) {
@@ -905,6 +1203,47 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
                                                  : make_quant_consts(bits, had_block, trust_factor);
     if (grid_kind == GRID_FP4 && cols % 32 != 0) return QUEST_ERR_SHAPE;
     const int cb = container_bits(bits);
+    if (dtype == QUEST_BF16 && had_block == 128 && cols % 128 == 0 && trust_factor >= 1.0f) {
+        // one thread per rotation block, when every tensor of the call is stored densely and asks for codes,
+        // scales and mask (plus, optionally, the GEMM operand)
+        bool ok = true;
+        for (int j = 0; j < njobs; ++j) {
+            const QuantJob &q = jobs[j];
+            if (q.rows == 0) continue;
+            if (!(q.codes && q.scales && q.mask) || q.rowsum || q.rot || q.cbf || q.ld != cols) ok = false;
+            if (grid_kind == GRID_FP4 && q.op8) ok = false;
+            if (reinterpret_cast<uintptr_t>(q.mask) % 16 != 0 || (q.op8 && reinterpret_cast<uintptr_t>(q.op8) % 16 != 0)) ok = false;
+        }
+        if (ok) {
+            const int T = (int)(cols / 128);
+            const int R = T >= 128 ? 1 : 128 / T;                       // rows per CTA: up to 128 threads
+            const int threads = (R * T + 31) / 32 * 32;
+            const size_t smem = (size_t)(threads / 32) * BLK_TILE_BYTES + sizeof(float) * (size_t)(threads + R);
+            for (int j0 = 0; j0 < njobs; j0 += 2) {
+                QuantArgs a;
+                int nb[2] = {0, 0};
+                for (int j = 0; j < 2; ++j) {
+                    QuantTensor &t = a.t[j];
+                    t = QuantTensor{nullptr, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+                    if (j0 + j < njobs) {
+                        const QuantJob &q = jobs[j0 + j];
+                        t.x = q.x; t.rows = q.rows; t.ld = q.ld; t.codes = q.codes; t.scales = q.scales;
+                        t.mask = q.mask; t.op8 = q.op8;
+                        nb[j] = (int)((q.rows + R - 1) / R);
+                    }
+                }
+                if (nb[0] + nb[1] == 0) continue;
+                a.blocks0 = nb[0];
+                a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = T; a.R = R;
+                a.inv_sqrt_g = 1.0f / sqrtf((float)had_block);
+                const dim3 grid((unsigned)(nb[0] + nb[1]));
+                const cudaError_t e = grid_kind == GRID_FP4 ? launch_block128<GRID_FP4>(cb, grid, threads, smem, st, a)
+                                                            : launch_block128<GRID_UNIFORM>(cb, grid, threads, smem, st, a);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
+            return QUEST_OK;
+        }
+    }
     if (cols % 32 == 0) {
         // 32 elements per thread (64 registers, twice the resident warps) for bfloat16 rows up to 8192 elements;
         // wider rows keep 64 per thread
