@@ -175,6 +175,43 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * quest_mlp_fwd -- forward pass of a Llama-style MLP block (the model family of the paper's experiments;
+ * hyper-parameter table: MLP width 8/3 of the hidden size) in which each of the three linear layers is
+ * Algorithm 1:
+ *
+ *     gate = QuEST_linear(x, w_gate);  up = QuEST_linear(x, w_up);     x is rotated and quantized once
+ *     h    = bf16( silu(gate) * up ),  silu(z) = z / (1 + exp(-z))     gate, up and the product in binary32
+ *     y    = QuEST_linear(h, w_down)
+ *
+ * Four launches on `stream`: quantizer (x, w_gate, w_up), contraction of x_q with both weight matrices with
+ * the SwiGLU in its epilogue (gate and up never reach memory; Section 5 fuses the dequantisation into the
+ * matmul epilogue for the same reason), quantizer (h, w_down), contraction with the dequantising epilogue.
+ * No allocation and no synchronisation, so the call can be captured into a CUDA graph.
+ *
+ *   x [T x H], w_gate [I x H], w_up [I x H], w_down [H x I]   device, dense row-major, `dtype`
+ *   T, H, I          tokens, hidden size, MLP width; H and I multiples of 32 (and of had_block), <= 16384
+ *   h [T x I]        device out, bfloat16, dense, 16-byte aligned: the hidden activations the down projection
+ *                    quantizes (a backward pass needs them as well)
+ *   y [T x H]        device out, dense, y_dtype
+ *   saved            device out: codes, per-row scales and trust masks of all five quantized tensors (what
+ *                    Algorithm 1 returns for each layer); codes and scales are required, masks may be NULL
+ *   workspace        device scratch of at least quest_mlp_workspace_bytes(T, H, I) bytes, 256-byte aligned
+ * Errors as for quest_linear_fwd.
+ */
+typedef struct quest_mlp_saved {
+    uint8_t *xq;  float *sx;  uint8_t *mx;      /* x       [T x H] */
+    uint8_t *wgq; float *swg; uint8_t *mwg;     /* w_gate  [I x H] */
+    uint8_t *wuq; float *swu; uint8_t *mwu;     /* w_up    [I x H] */
+    uint8_t *hq;  float *sh;  uint8_t *mh;      /* h       [T x I] */
+    uint8_t *wdq; float *swd; uint8_t *mwd;     /* w_down  [H x I] */
+} quest_mlp_saved;
+int quest_mlp_fwd(const void *x, const void *w_gate, const void *w_up, const void *w_down, int dtype,
+                  int64_t T, int64_t H, int64_t I, int bits, int had_block, float trust_factor,
+                  void *h, void *y, int y_dtype, const quest_mlp_saved *saved,
+                  void *workspace, size_t workspace_bytes, void *stream);
+size_t quest_mlp_workspace_bytes(int64_t T, int64_t H, int64_t I);
+
+/*
  * quest_linear_bwd -- Algorithm 2 (QuEST training backward) for one linear layer, from what
  * quest_linear_fwd saved:
  *

@@ -240,6 +240,55 @@ def quest_linear_bwd(dy: torch.Tensor, fwd: dict, bits: int, had_block: int, K: 
     return {"dx": dx, "dw": dw}
 
 
+# ---- MLP block: gate / up / SwiGLU / down, every linear layer Algorithm 1 -------------------------
+
+class _MlpSaved(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("xq", "sx", "mx", "wgq", "swg", "mwg", "wuq", "swu", "mwu",
+                                               "hq", "sh", "mh", "wdq", "swd", "mwd")]
+
+
+def quest_mlp_workspace_bytes(T: int, H: int, I: int) -> int:
+    return int(_lib.load().quest_mlp_workspace_bytes(T, H, I))
+
+
+def mlp_buffers(T: int, H: int, I: int, bits: int, device=None, out_dtype=torch.bfloat16, want_masks: bool = True) -> dict:
+    """Every output of ``quest_mlp_fwd`` and its workspace, allocated once (the call itself allocates nothing)."""
+    dev = device or torch.device("cuda")
+    cb = container_bits(bits)
+    n = quest_mlp_workspace_bytes(T, H, I)
+    if n == 0:
+        raise ValueError("quest_mlp_fwd: unsupported shape (H, I multiples of 32, at most 16384)")
+    u8 = lambda *s: torch.empty(s, dtype=torch.uint8, device=dev)
+    f32 = lambda *s: torch.empty(s, dtype=torch.float32, device=dev)
+    b = {"h": torch.empty((T, I), dtype=torch.bfloat16, device=dev), "y": torch.empty((T, H), dtype=out_dtype, device=dev),
+         "xq": u8(T, H * cb // 8), "sx": f32(T), "wgq": u8(I, H * cb // 8), "swg": f32(I), "wuq": u8(I, H * cb // 8),
+         "swu": f32(I), "hq": u8(T, I * cb // 8), "sh": f32(T), "wdq": u8(H, I * cb // 8), "swd": f32(H),
+         "workspace": u8(n), "launches": 4}
+    for k, shape in (("mx", (T, H // 8)), ("mwg", (I, H // 8)), ("mwu", (I, H // 8)), ("mh", (T, I // 8)), ("mwd", (H, I // 8))):
+        b[k] = u8(*shape) if want_masks else None
+    return b
+
+
+def quest_mlp_fwd(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor, w_down: torch.Tensor, bits: int,
+                  had_block: int, trust_factor: float = 1.0, buffers: dict = None, out_dtype=torch.bfloat16) -> dict:
+    """y = down(silu(gate(x)) * up(x)) with QuEST linear layers.  Returns the ``buffers`` dict: "y" [T, H],
+    "h" [T, I] bfloat16 and the codes / scales / masks of x, w_gate, w_up, h, w_down."""
+    _require_cuda(x, w_gate, w_up, w_down)
+    T, H = x.shape
+    I = w_gate.shape[0]
+    if w_up.shape != (I, H) or w_down.shape != (H, I) or not all(t.is_contiguous() for t in (x, w_gate, w_up, w_down)):
+        raise ValueError("quest_mlp_fwd: x [T, H], w_gate / w_up [I, H], w_down [H, I], all contiguous")
+    if not (x.dtype == w_gate.dtype == w_up.dtype == w_down.dtype):
+        raise TypeError("quest_mlp_fwd: x and the weights share one dtype")
+    b = buffers if buffers is not None else mlp_buffers(T, H, I, bits, x.device, out_dtype)
+    sv = _MlpSaved(*[(b[n].data_ptr() if b.get(n) is not None else None) for n, _ in _MlpSaved._fields_])
+    st = _lib.load().quest_mlp_fwd(_p(x), _p(w_gate), _p(w_up), _p(w_down), _dtype_code(x), T, H, I, bits, had_block,
+                                   ctypes.c_float(trust_factor), _p(b["h"]), _p(b["y"]), _dtype_code(b["y"]),
+                                   ctypes.byref(sv), _p(b["workspace"]), b["workspace"].numel(), _stream())
+    _lib.check(st)
+    return b
+
+
 # ---- weight-only variant (Section 4.5): b-bit weights, bfloat16 activations -----------------------
 
 def quest_weight_only_workspace_bytes(M: int, N: int, K: int) -> int:

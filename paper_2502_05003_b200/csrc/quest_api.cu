@@ -321,6 +321,92 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
     return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits, bits, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);
 }
 
+// ---- MLP block: three Algorithm-1 layers with the SwiGLU fused into the first contraction -------
+
+namespace {
+struct MlpWorkspace {
+    int8_t *b_gu; int32_t *rs_gu;     // operands of w_gate rows [0, I) and w_up rows [I, 2I), K = H
+    int8_t *a_x;  int32_t *rs_x;      // operand of x [T x H]
+    int8_t *b_d;  int32_t *rs_d;      // operand of w_down [H x I]
+    int8_t *a_h;  int32_t *rs_h;      // operand of h [T x I]
+    size_t bytes;
+};
+MlpWorkspace carve_mlp(void *base, int64_t T, int64_t H, int64_t I) {
+    MlpWorkspace w;
+    uint8_t *b = reinterpret_cast<uint8_t *>(base);
+    size_t off = 0;
+    auto take = [&](size_t n) { uint8_t *p = b + off; off += align_up(n, 256); return p; };
+    w.b_gu = reinterpret_cast<int8_t *>(take((size_t)(2 * I * H)));
+    w.rs_gu = reinterpret_cast<int32_t *>(take((size_t)(2 * I) * 4));
+    w.a_x = reinterpret_cast<int8_t *>(take((size_t)(T * H)));
+    w.rs_x = reinterpret_cast<int32_t *>(take((size_t)T * 4));
+    w.b_d = reinterpret_cast<int8_t *>(take((size_t)(H * I)));
+    w.rs_d = reinterpret_cast<int32_t *>(take((size_t)H * 4));
+    w.a_h = reinterpret_cast<int8_t *>(take((size_t)(T * I)));
+    w.rs_h = reinterpret_cast<int32_t *>(take((size_t)T * 4));
+    w.bytes = off;
+    return w;
+}
+}  // namespace
+
+size_t quest_mlp_workspace_bytes(int64_t T, int64_t H, int64_t I) {
+    if (validate_gemm_shape(T, I, H, 1, 1) != QUEST_OK || validate_gemm_shape(T, H, I, 1, 1) != QUEST_OK) return 0;
+    if (H > 16384 || I > 16384) return 0;
+    return carve_mlp(nullptr, T, H, I).bytes;
+}
+
+int quest_mlp_fwd(const void *x, const void *w_gate, const void *w_up, const void *w_down, int dtype,
+                  int64_t T, int64_t H, int64_t I, int bits, int had_block, float trust_factor,
+                  void *h, void *y, int y_dtype, const quest_mlp_saved *sv,
+                  void *workspace, size_t workspace_bytes, void *stream) {
+    if (!x || !w_gate || !w_up || !w_down || !h || !y || !sv) return QUEST_ERR_NULL;
+    if (!sv->xq || !sv->sx || !sv->wgq || !sv->swg || !sv->wuq || !sv->swu || !sv->hq || !sv->sh || !sv->wdq || !sv->swd)
+        return QUEST_ERR_NULL;
+    if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+    int s = validate_gemm_shape(T, I, H, bits, bits);
+    if (s) return s;
+    if ((s = validate_gemm_shape(T, H, I, bits, bits))) return s;
+    if ((s = validate_quantize(x, dtype, T, H, H, bits, had_block, trust_factor, sv->xq, sv->mx))) return s;
+    if ((s = validate_quantize(w_gate, dtype, I, H, H, bits, had_block, trust_factor, sv->wgq, sv->mwg))) return s;
+    if ((s = validate_quantize(w_up, dtype, I, H, H, bits, had_block, trust_factor, sv->wuq, sv->mwu))) return s;
+    if ((s = validate_quantize(h, QUEST_BF16, T, I, I, bits, had_block, trust_factor, sv->hq, sv->mh))) return s;
+    if ((s = validate_quantize(w_down, dtype, H, I, I, bits, had_block, trust_factor, sv->wdq, sv->mwd))) return s;
+    if (!aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_mlp_workspace_bytes(T, H, I))
+        return QUEST_ERR_WORKSPACE;
+    if (T == 0) return QUEST_OK;
+    if ((s = check_device())) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    MlpWorkspace ws = carve_mlp(workspace, T, H, I);
+    const bool rs = bits == 8;
+    const size_t up_off = (size_t)I * (size_t)(e2m1_operands(bits, bits) ? H / 2 : H);   // operand bytes of the gate rows
+    {
+        StageScope scope(QUEST_STAGE_QUANT_X, st);
+        const QuantJob jobs[3] = {{x, T, H, sv->xq, sv->sx, sv->mx, ws.a_x, rs ? ws.rs_x : nullptr},
+                                  {w_gate, I, H, sv->wgq, sv->swg, sv->mwg, ws.b_gu, rs ? ws.rs_gu : nullptr},
+                                  {w_up, I, H, sv->wuq, sv->swu, sv->mwu, ws.b_gu + up_off, rs ? ws.rs_gu + I : nullptr}};
+        if ((s = launch_quantize(jobs, 3, dtype, H, bits, had_block, trust_factor, st))) return s;
+    }
+    {
+        StageScope scope(QUEST_STAGE_GEMM, st);
+        if ((s = launch_gemm_swiglu(ws.a_x, ws.b_gu, ws.rs_x, ws.rs_gu, bits, sv->sx, sv->swg, sv->swu, T, I, H, h, st))) return s;
+    }
+    {
+        StageScope scope(QUEST_STAGE_QUANT_W, st);
+        const QuantJob jh = {h, T, I, sv->hq, sv->sh, sv->mh, ws.a_h, rs ? ws.rs_h : nullptr};
+        const QuantJob jd = {w_down, H, I, sv->wdq, sv->swd, sv->mwd, ws.b_d, rs ? ws.rs_d : nullptr};
+        if (dtype == QUEST_BF16) {
+            const QuantJob jobs[2] = {jh, jd};
+            if ((s = launch_quantize(jobs, 2, QUEST_BF16, I, bits, had_block, trust_factor, st))) return s;
+        } else {
+            if ((s = launch_quantize(&jh, 1, QUEST_BF16, I, bits, had_block, trust_factor, st))) return s;
+            if ((s = launch_quantize(&jd, 1, dtype, I, bits, had_block, trust_factor, st))) return s;
+        }
+    }
+    StageScope scope(QUEST_STAGE_GEMM, st);
+    return launch_gemm(ws.a_h, ws.b_d, ws.rs_h, ws.rs_d, bits, bits, sv->sh, sv->swd, T, H, I, y, y_dtype, H, nullptr, st);
+}
+
 // ---- FP4 (E2M1) grid variant (Section 4.4, "The FP4 Format") -----------------------------------
 
 float quest_alpha_star_fp4(void) { return alpha_star_fp4(); }

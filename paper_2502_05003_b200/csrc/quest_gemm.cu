@@ -68,6 +68,10 @@ struct GemmParams {
     int32_t *acc;
     const uint8_t *mask;   // backward mode: trust-mask bitmap of the output, [M x N/8] bytes (1 = keep)
     int *status;
+    // SwiGLU mode: the B operand holds the gate rows [0, N) and, from row up_row0 on, the up rows; sw / rs_b
+    // index the gate rows, sw2 the up rows (rs_b is one array over all rows of B)
+    const float *sw2;
+    int up_row0;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -317,7 +321,12 @@ struct SmemLayout {
 // OPL (bfloat16 modes only): 0 = both operands K-major; 1 = B MN-major (its memory rows run along the
 // contraction); 2 = A and B MN-major.  The backward pass uses 1 and 2 to read dy and the dequantised
 // operands as they lie in memory, without transposed copies.
-template <int BN, int MODE, bool TWO, bool YT, int OPL = 0>
+// SWIGLU (integer modes 0, 1, 5 with BN = 256 and the TMA-store epilogue): the 256 accumulator columns
+// of a tile are 128 columns of the gate projection followed by the SAME 128 columns of the up
+// projection (the B operand stacks the rows of w_gate and w_up), every epilogue thread holds gate and
+// up of 64 output columns of its row, and the tile leaves as h = silu(gate) * up in bfloat16: the
+// MLP block's gate and up products never reach memory.
+template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
@@ -333,6 +342,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr bool AMN = OPL == 2, BMN = OPL >= 1;
     static_assert(OPL == 0 || MODE == 2 || MODE == 3, "MN-major operands: bfloat16 backward modes only");
     static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
+    static_assert(!SWIGLU || (BN == 256 && YT && (MODE == 0 || MODE == 1 || MODE == 5)), "SwiGLU epilogue: integer modes, 256 columns, TMA stores");
+    constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
     constexpr int STAGES = L::NSTAGES;
     constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
     extern __shared__ uint8_t smem_raw[];
@@ -406,7 +417,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     pdl_wait();     // set-up above overlaps the previous kernel; operands and outputs are touched only from here
 
     const int num_m = (p.M + TILE_M - 1) / TILE_M;
-    const int num_n = (p.N + BN - 1) / BN;
+    const int num_n = (p.N + BN_OUT - 1) / BN_OUT;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
 
@@ -419,7 +430,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 int tm, tn;
                 tile_coords(tile, num_m, num_n, tm, tn);
                 const int m0 = tm * TILE_M + (int)rank * BM;                     // this CTA's rows of A
-                const int n0 = tn * BN + (int)rank * L::B_ROWS;                  // this CTA's rows of B
+                // this CTA's rows of B (SwiGLU pair: the leader stages the gate rows, its peer the up rows)
+                const int n0 = SWIGLU ? tn * BN_OUT + (int)rank * p.up_row0 : tn * BN + (int)rank * L::B_ROWS;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, p.status, ST_PRODUCER);
                     if (!ok) break;
@@ -458,6 +470,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                             for (int c = 0; c < L::B_ROWS / 64; ++c)
                                 tma_load_2d(smem_u32(sa + L::A_BYTES + c * 8192), &tmB, (n0 + 64 * c) * 2, kb * 64, fb);
+                        } else if constexpr (SWIGLU) {         // two boxes of 128 rows: gate rows, then up rows
+                            tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
+                            tma_load_2d(smem_u32(sa + L::A_BYTES + (BN / 2) * BK), &tmB, kb * BK, n0 + p.up_row0, fb);
                         } else {
                             tma_load_2d(smem_u32(sa + L::A_BYTES), &tmB, kb * BK, n0, fb);
                         }
@@ -532,7 +547,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         //      and the column half (w - 2) / 4 of the tile ------------------------------------------------
         constexpr int CW = BN / 2;                     // columns per warp
         const int quarter = warp & 3;
-        const int cbase = ((warp - 2) >> 2) * CW;
+        const int hgrp = (warp - 2) >> 2;              // which half of the tile's (output) columns
+        const int cbase = hgrp * CW;
+        // accumulator column of this warp's chunk c0 (0, 32, 64, 96): plain modes take CW consecutive columns;
+        // SwiGLU takes gate columns [64 hgrp, +64) and the up columns of the same outputs, 128 further on
+        auto acc_col = [&](int c0) { return SWIGLU ? (c0 < 64 ? 64 * hgrp + c0 : 128 + 64 * hgrp + (c0 - 64)) : cbase + c0; };
         const int ep_tid = threadIdx.x - 64;           // 0..255 over the epilogue warps
         int t = 0;
         bool ok = true;
@@ -546,7 +565,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int tm, tn;
             tile_coords(tile, num_m, num_n, tm, tn);
             const int m0 = tm * TILE_M + (int)rank * BM;
-            const int n0 = tn * BN;
+            const int n0 = tn * BN_OUT;
             const int buf = NBUF == 2 ? (t & 1) : 0;
             const uint32_t bphase = (uint32_t)(NBUF == 2 ? (t >> 1) : t) & 1u;
             // stage this tile's column scales (and column corrections) in shared memory; the
@@ -555,9 +574,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float *swt = sw_tile + (t & 1) * BN;
             int32_t *cbt = cb_tile + (t & 1) * BN;
             for (int c = ep_tid; c < BN; c += 32 * EPI_WARPS) {
-                const int col = n0 + c;
-                if (!BWD) swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
-                if (CORR) cbt[c] = (p.rs_b && col < p.N) ? p.cb * __ldg(p.rs_b + col) : 0;
+                if constexpr (SWIGLU) {
+                    const bool up = c >= BN_OUT;
+                    const int col = n0 + (up ? c - BN_OUT : c);
+                    swt[c] = col < p.N ? __ldg((up ? p.sw2 : p.sw) + col) : 0.0f;
+                    if (CORR) cbt[c] = (p.rs_b && col < p.N) ? p.cb * __ldg(p.rs_b + col + (up ? p.up_row0 : 0)) : 0;
+                } else {
+                    const int col = n0 + c;
+                    if (!BWD) swt[c] = (p.y && col < p.N) ? __ldg(p.sw + col) : 0.0f;
+                    if (CORR) cbt[c] = (p.rs_b && col < p.N) ? p.cb * __ldg(p.rs_b + col) : 0;
+                }
             }
             const int row = m0 + quarter * 32 + lane;
             const bool row_ok = row < p.M;
@@ -587,11 +613,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tc_fence_after();
             // all of this warp's accumulator columns in one go, then hand the TMEM buffer back to
             // the MMA warp before any arithmetic
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cbase);
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
             uint32_t r[CW];
 #pragma unroll
-            for (int c0 = 0; c0 < CW; c0 += 32)
-                if (n0 + cbase + c0 < p.N) tmem_ld32_issue(t_row + (uint32_t)c0, &r[c0]);     // uniform predicate
+            for (int c0 = 0; c0 < CW; c0 += 32) {
+                const int first_out = SWIGLU ? n0 + 64 * hgrp + (c0 & 63) : n0 + cbase + c0;
+                if (first_out < p.N) tmem_ld32_issue(t_row + (uint32_t)acc_col(c0), &r[c0]);     // uniform predicate
+            }
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < CW; ++j) pin(r[j]);
@@ -633,8 +661,77 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
+            if constexpr (SWIGLU) {
+                const int out0 = n0 + 64 * hgrp;               // first of this thread's 64 output columns
+                if (out0 < p.N) {                              // uniform across the warp
+                    const float2 sx2 = make_float2(sxr, sxr);
 #pragma unroll
-            for (int c0 = 0; c0 < CW; c0 += 32) {
+                    for (int c0 = 0; c0 < CW; c0 += 32) {
+                        uint32_t *rc = &r[c0];
+                        const int ac = acc_col(c0);
+                        if (n0 + 64 * hgrp + (c0 & 63) < p.N) {
+                            if (CORR) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    rc[j] = (uint32_t)((int32_t)((uint32_t)p.mul * rc[j] + (uint32_t)rsa + (uint32_t)cbt[ac + j]) >> p.sh);
+                            }
+                            const float2 *sw2 = reinterpret_cast<const float2 *>(swt + ac);
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) {
+                                const float2 a2 = MX ? make_float2(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]))
+                                                     : make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
+                                const float2 y2 = __fmul2_rn(__fmul2_rn(sx2, sw2[j >> 1]), a2);
+                                rc[j] = __float_as_uint(y2.x);
+                                rc[j + 1] = __float_as_uint(y2.y);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) rc[j] = 0u;
+                        }
+                    }
+                    // h = silu(gate) * up, silu(z) = z / (1 + exp(-z)); one rounding to bfloat16.  The exponential and
+                    // the reciprocal are the hardware approximations (a few units of 2^-23 each, no branches):
+                    // exp(-z) overflows to +inf for z < -88, where the quotient is -0 as it should be.
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) {
+                        const float g = __uint_as_float(r[j]), u = __uint_as_float(r[64 + j]);
+                        float e, rc;
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(g * -1.4426950408889634f));
+                        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(1.0f + e));
+                        r[j] = __float_as_uint((g * rc) * u);
+                    }
+                    uint8_t *slab = slab_base;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
+                    uint8_t *rowp = slab + lane * 128;
+                    const int sw7 = lane & 7;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint4 q;
+                        __nv_bfloat162 hh;
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1]));
+                        q.x = *reinterpret_cast<uint32_t *>(&hh);
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
+                        q.y = *reinterpret_cast<uint32_t *>(&hh);
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
+                        q.z = *reinterpret_cast<uint32_t *>(&hh);
+                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
+                        q.w = *reinterpret_cast<uint32_t *>(&hh);
+                        *reinterpret_cast<uint4 *>(rowp + ((j ^ sw7) << 4)) = q;
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile(
+                            "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                            ::"l"(reinterpret_cast<uint64_t>(&tmY)), "r"(smem_u32(slab)), "r"(out0 * 2), "r"(m0 + quarter * 32)
+                            : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                }
+            }
+#pragma unroll
+            for (int c0 = 0; c0 < (SWIGLU ? 0 : CW); c0 += 32) {
                 const int col0 = n0 + cbase + c0;
                 if (col0 < p.N) {                      // uniform across the warp
                     const bool full = col0 + 32 <= p.N;
@@ -953,20 +1050,21 @@ int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes
     return QUEST_OK;
 }
 
-template <int BN, int MODE, bool TWO, bool YT, int OPL = 0>
+template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
                    cudaStream_t st) {
     using L = SmemLayout<BN, TWO>;
     static DynamicSmemOnce smem_attr;            // per kernel instantiation, per device
     {
-        cudaError_t e = smem_attr.set(gemm_i8_kernel<BN, MODE, TWO, YT, OPL>, L::TOTAL);
+        cudaError_t e = smem_attr.set(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU>, L::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int tile_m = TWO ? 2 * BM : BM;
-    const int tiles = ((p.M + tile_m - 1) / tile_m) * ((p.N + BN - 1) / BN);
+    const int bn_out = SWIGLU ? BN / 2 : BN;
+    const int tiles = ((p.M + tile_m - 1) / tile_m) * ((p.N + bn_out - 1) / bn_out);
     int grid;
     if (TWO) {
         const int pairs = tiles < sms / 2 ? tiles : sms / 2;
@@ -974,7 +1072,7 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
     } else {
         grid = tiles < sms ? tiles : sms;
     }
-    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT, OPL>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
+    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
                                TWO ? 2 : 1, tmA, tmB, tmY, p);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
@@ -1064,7 +1162,7 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
     else { p.mul = 2; p.ca = 1; p.cb = 0; p.ck = 0; p.sh = 7 - bits_x; }
     p.rs_a = p.ca ? rs_a : nullptr;                      // row sums of the x operand bytes
     p.rs_b = p.cb ? rs_b : nullptr;                      // row sums of the w operand bytes
-    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr; p.sw2 = nullptr; p.up_row0 = 0;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
 
@@ -1095,6 +1193,39 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
 #undef QUEST_GEMM
 }
 
+// Gate and up projections of an MLP block with the SwiGLU fused into the epilogue:
+//   h[i][j] = bf16( silu(sx[i] sw_gate[j] acc_g[i][j]) * (sx[i] sw_up[j] acc_u[i][j]) ),  j < I,
+// where b8 stacks the operand rows of w_gate ([0, I)) and w_up ([I, 2I)) and rs_b their row sums.
+int launch_gemm_swiglu(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const int32_t *rs_b, int bits,
+                       const float *sx, const float *sw_gate, const float *sw_up, int64_t M, int64_t I, int64_t K,
+                       void *h, cudaStream_t st) {
+    if (M == 0 || I == 0) return QUEST_OK;
+    const bool mx = e2m1_operands(bits, bits), b8x = bits == 8;
+    GemmParams p;
+    p.M = (int)M; p.N = (int)I; p.K = (int)(mx ? K / 2 : K);
+    p.sx = sx; p.sw = sw_gate; p.sw2 = sw_up; p.up_row0 = (int)I;
+    if (mx) { p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0; }
+    else if (b8x) { p.mul = 4; p.ca = 2; p.cb = 2; p.ck = (int)K; p.sh = 0; }
+    else { p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 14 - 2 * bits; }
+    p.rs_a = b8x ? rs_a : nullptr; p.rs_b = b8x ? rs_b : nullptr;
+    p.y = h; p.y_dtype = QUEST_BF16; p.ldy = I; p.acc = nullptr; p.mask = nullptr;
+    p.status = device_status_word();
+    if (!p.status) return QUEST_ERR_CUDA;
+    const bool pair = M > 128;
+    CUtensorMap tmA, tmB, tmY;
+    int s = make_operand_map(&tmA, a8, M, p.K, BM);
+    if (s) return s;
+    if ((s = make_operand_map(&tmB, b8, 2 * I, p.K, 128))) return s;       // boxes of 128 rows: gate rows or up rows
+    if ((s = make_output_map(&tmY, h, M, I * 2, I * 2))) return s;
+#define QUEST_GEMM_SG(MODEV) \
+    (pair ? launch_gemm_bn<256, MODEV, true, true, 0, true>(tmA, tmB, tmY, p, st) \
+          : launch_gemm_bn<256, MODEV, false, true, 0, true>(tmA, tmB, tmY, p, st))
+    if (mx) return QUEST_GEMM_SG(5);
+    if (b8x) return QUEST_GEMM_SG(1);
+    return QUEST_GEMM_SG(0);
+#undef QUEST_GEMM_SG
+}
+
 // Backward-pass contraction (the two products of Algorithm 2): out[i][j] = mask[i][j] * sum_k A(i, k) B(j, k) with
 // bfloat16 operands and binary32 output [I x J].  `opl` says how the operands lie in memory:
 //   0: a [I x Kc], b [J x Kc], the contraction index contiguous (K-major);
@@ -1109,7 +1240,7 @@ int launch_gemm_bf16_masked(const void *a, const void *b, int64_t I, int64_t J, 
     p.M = (int)I; p.N = (int)J; p.K = (int)(2 * Kc);
     p.sx = nullptr; p.sw = nullptr; p.rs_a = nullptr; p.rs_b = nullptr;
     p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
-    p.y = out; p.y_dtype = out_dtype; p.ldy = J; p.acc = nullptr; p.mask = mask;
+    p.y = out; p.y_dtype = out_dtype; p.ldy = J; p.acc = nullptr; p.mask = mask; p.sw2 = nullptr; p.up_row0 = 0;
     const int64_t esz = out_dtype == QUEST_F32 ? 4 : 2;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
@@ -1150,7 +1281,7 @@ int launch_gemm_e2m1(const uint8_t *xq, const uint8_t *wq, const float *sx, cons
     p.M = (int)M; p.N = (int)N; p.K = (int)(K / 2);
     p.sx = sx; p.sw = sw; p.rs_a = nullptr; p.rs_b = nullptr;
     p.mul = acc_mul; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
-    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = acc; p.mask = nullptr; p.sw2 = nullptr; p.up_row0 = 0;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
     const bool wide = N > 128;
@@ -1182,7 +1313,7 @@ int launch_gemm_bf16_scaled(const void *a, const void *b, const float *sw, int64
     p.M = (int)M; p.N = (int)N; p.K = (int)(2 * K);
     p.sx = nullptr; p.sw = sw; p.rs_a = nullptr; p.rs_b = nullptr;
     p.mul = 1; p.ca = 0; p.cb = 0; p.ck = 0; p.sh = 0;
-    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = nullptr; p.mask = nullptr;
+    p.y = y; p.y_dtype = y_dtype; p.ldy = ldy; p.acc = nullptr; p.mask = nullptr; p.sw2 = nullptr; p.up_row0 = 0;
     p.status = device_status_word();
     if (!p.status) return QUEST_ERR_CUDA;
     const bool wide = N > 128;

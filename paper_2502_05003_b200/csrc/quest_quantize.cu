@@ -163,8 +163,10 @@ struct QuantTensor {
     uint16_t *rot;         // bfloat16 of the orthonormal rotation itself (weight-only variant)
     uint16_t *cbf;         // grid values c = 2k - (2^b - 1) as bfloat16 (weight-only variant)
 };
+constexpr int MAX_QUANT_TENSORS = 4;   // tensors one launch of the block kernel can serve (the other kernels: two)
 struct QuantArgs {
-    QuantTensor t[2];
+    QuantTensor t[MAX_QUANT_TENSORS];
+    int bend[MAX_QUANT_TENSORS];        // block kernel: CTAs [bend[j-1], bend[j]) work on tensor j
     int blocks0;
     int cols, bits, had_block;
     QuantConsts qc;
@@ -932,9 +934,10 @@ quantize_block128_kernel(const __grid_constant__ QuantArgs a) {
     pdl_launch_dependents();
     pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-    const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
+    const int bid = (int)blockIdx.x;
+    const int which = (bid >= a.bend[0] ? 1 : 0) + (bid >= a.bend[1] ? 1 : 0) + (bid >= a.bend[2] ? 1 : 0);
     const QuantTensor &tn = a.t[which];
-    const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
+    const int blk = which ? bid - a.bend[which - 1] : bid;
     const int cols = a.cols;
     const int T = cols >> 7;                                   // blocks (= threads) per row
     const long long row0 = (long long)blk * a.R;
@@ -1219,24 +1222,25 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             const int R = T >= 128 ? 1 : 128 / T;                       // rows per CTA: up to 128 threads
             const int threads = (R * T + 31) / 32 * 32;
             const size_t smem = (size_t)(threads / 32) * BLK_TILE_BYTES + sizeof(float) * (size_t)(threads + R);
-            for (int j0 = 0; j0 < njobs; j0 += 2) {
+            for (int j0 = 0; j0 < njobs; j0 += MAX_QUANT_TENSORS) {
                 QuantArgs a;
-                int nb[2] = {0, 0};
-                for (int j = 0; j < 2; ++j) {
+                int total = 0;
+                for (int j = 0; j < MAX_QUANT_TENSORS; ++j) {
                     QuantTensor &t = a.t[j];
                     t = QuantTensor{nullptr, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
                     if (j0 + j < njobs) {
                         const QuantJob &q = jobs[j0 + j];
                         t.x = q.x; t.rows = q.rows; t.ld = q.ld; t.codes = q.codes; t.scales = q.scales;
                         t.mask = q.mask; t.op8 = q.op8;
-                        nb[j] = (int)((q.rows + R - 1) / R);
+                        total += (int)((q.rows + R - 1) / R);
                     }
+                    a.bend[j] = total;
                 }
-                if (nb[0] + nb[1] == 0) continue;
-                a.blocks0 = nb[0];
+                if (total == 0) continue;
+                a.blocks0 = a.bend[0];
                 a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = T; a.R = R;
                 a.inv_sqrt_g = 1.0f / sqrtf((float)had_block);
-                const dim3 grid((unsigned)(nb[0] + nb[1]));
+                const dim3 grid((unsigned)total);
                 const cudaError_t e = grid_kind == GRID_FP4 ? launch_block128<GRID_FP4>(cb, grid, threads, smem, st, a)
                                                             : launch_block128<GRID_UNIFORM>(cb, grid, threads, smem, st, a);
                 if (e != cudaSuccess) return cuda_fail(e);
@@ -1277,6 +1281,9 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             }
             if (nb[0] + nb[1] == 0) continue;
             a.blocks0 = nb[0];
+            for (int j = 0; j < MAX_QUANT_TENSORS; ++j) a.bend[j] = j == 0 ? nb[0] : nb[0] + nb[1];
+            for (int j = 2; j < MAX_QUANT_TENSORS; ++j)
+                a.t[j] = QuantTensor{nullptr, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
             a.cols = (int)cols; a.bits = bits; a.had_block = had_block; a.qc = qc; a.S = S; a.R = R;
             a.inv_sqrt_g = 1.0f / sqrtf((float)had_block);
             const dim3 grid((unsigned)(nb[0] + nb[1]));

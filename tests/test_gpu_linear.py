@@ -67,9 +67,10 @@ def test_config3(bits, trust):
     check_linear(c["x"], c["w"], bits, 128, trust, torch.bfloat16, BF16_OUT_RTOL, sample_rows=rows)
 
 
-def test_config4_mlp_block():
-    """gate/up -> SwiGLU (harness glue in torch) -> down; the oracle for the down projection is
-    fed the GPU's own bf16 hidden activations."""
+def test_config4_layers_one_call_each():
+    """The three layers of config 4 as separate quest_linear_fwd calls with the SwiGLU as torch glue (the
+    fused block is tested in test_gpu_mlp.py); the oracle for the down projection is fed the GPU's own
+    bf16 hidden activations."""
     import paper_2502_05003_b200 as quest
     c = synth.config4()
     rows = np.random.default_rng(2).choice(8192, 64, replace=False)
