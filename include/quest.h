@@ -175,6 +175,23 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * quest_linear_fwd in two calls, for callers that schedule the two halves of Algorithm 1 themselves (weights
+ * quantized once and contracted with several batches of activations; a half run on another stream; a half timed
+ * alone).  quest_linear_fwd_quantize is the rotation and projection steps: it writes the codes, scales and masks
+ * exactly as quest_linear_fwd does (same arguments, without y) and leaves the tensor-core operands of x and w in
+ * `workspace`.  quest_linear_fwd_contract is the product step: it contracts the operands that the first call left
+ * in the same `workspace` (same M, N, K, bits; nothing else may have written the workspace in between) and applies
+ * the scales.  The pair, in this order on one stream, is quest_linear_fwd.
+ */
+int quest_linear_fwd_quantize(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                              int bits, int had_block, float trust_factor,
+                              uint8_t *xq, float *sx, uint8_t *mx,
+                              uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                              void *workspace, size_t workspace_bytes, void *stream);
+int quest_linear_fwd_contract(const float *sx, const float *sw, int64_t M, int64_t N, int64_t K, int bits,
+                              void *y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * quest_mlp_fwd -- forward pass of a Llama-style MLP block (the model family of the paper's experiments;
  * hyper-parameter table: MLP width 8/3 of the hidden size) in which each of the three linear layers is
  * Algorithm 1:

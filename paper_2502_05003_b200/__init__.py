@@ -209,6 +209,29 @@ def quest_linear_fwd(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int
     return out
 
 
+def quest_linear_fwd_quantize(x: torch.Tensor, w: torch.Tensor, bits: int, had_block: int, trust_factor: float,
+                              saved: dict, workspace: torch.Tensor) -> None:
+    """First half of ``quest_linear_fwd``: codes, scales, masks into ``saved`` (preallocated, keys xq, sx, mx, wq,
+    sw, mw) and the tensor-core operands into ``workspace``."""
+    _require_cuda(x, w, workspace)
+    M, K = x.shape
+    N = w.shape[0]
+    st = _lib.load().quest_linear_fwd_quantize(
+        _p(x), _p(w), _dtype_code(x), M, N, K, bits, had_block, ctypes.c_float(trust_factor),
+        _p(saved["xq"]), _p(saved["sx"]), _p(saved.get("mx")), _p(saved["wq"]), _p(saved["sw"]), _p(saved.get("mw")), 0,
+        _p(workspace), workspace.numel(), _stream())
+    _lib.check(st)
+
+
+def quest_linear_fwd_contract(saved: dict, M: int, N: int, K: int, bits: int, y: torch.Tensor, workspace: torch.Tensor) -> None:
+    """Second half of ``quest_linear_fwd``: the contraction of the operands that ``quest_linear_fwd_quantize`` left
+    in ``workspace``, scaled by ``saved["sx"]`` and ``saved["sw"]``, into ``y``."""
+    _require_cuda(y, workspace)
+    st = _lib.load().quest_linear_fwd_contract(_p(saved["sx"]), _p(saved["sw"]), M, N, K, bits, _p(y), _dtype_code(y),
+                                               _p(workspace), workspace.numel(), _stream())
+    _lib.check(st)
+
+
 def quest_bwd_workspace_bytes(M: int, N: int, K: int) -> int:
     return int(_lib.load().quest_bwd_workspace_bytes(M, N, K))
 

@@ -279,21 +279,19 @@ int quest_lowbit_gemm(const uint8_t *xq, const float *sx, int bits_x,
                        st);
 }
 
-int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
-                     int bits, int had_block, float trust_factor,
-                     void *y, int y_dtype,
-                     uint8_t *xq, float *sx, uint8_t *mx,
-                     uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
-                     void *workspace, size_t workspace_bytes, void *stream) {
-    if (!y || !xq || !sx || !wq || !sw) return QUEST_ERR_NULL;
+int quest_linear_fwd_quantize(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                              int bits, int had_block, float trust_factor,
+                              uint8_t *xq, float *sx, uint8_t *mx,
+                              uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                              void *workspace, size_t workspace_bytes, void *stream) {
+    if (!xq || !sx || !wq || !sw) return QUEST_ERR_NULL;
     if (!w_is_cached && !w) return QUEST_ERR_NULL;
     if (w_is_cached < 0 || w_is_cached > 2) return QUEST_ERR_SHAPE;
-    if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
     int s = validate_gemm_shape(M, N, K, bits, bits);
     if (s) return s;
     if ((s = validate_quantize(x, dtype, M, K, K, bits, had_block, trust_factor, xq, mx))) return s;
     if (!w_is_cached && (s = validate_quantize(w, dtype, N, K, K, bits, had_block, trust_factor, wq, mw))) return s;
-    if (!aligned(wq, 16) || !aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    if (!aligned(wq, 16)) return QUEST_ERR_ALIGN;
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, bits, bits))
         return QUEST_ERR_WORKSPACE;
     if ((s = check_device())) return s;
@@ -317,8 +315,39 @@ int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t
         const QuantJob jobs[2] = {jx, {w, N, K, wq, sw, mw, ws.b8, need_rs ? ws.rs_b : nullptr}};
         if ((s = launch_quantize(jobs, 2, dtype, K, bits, had_block, trust_factor, st))) return s;
     }
+    return QUEST_OK;
+}
+
+int quest_linear_fwd_contract(const float *sx, const float *sw, int64_t M, int64_t N, int64_t K, int bits,
+                              void *y, int y_dtype, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!y || !sx || !sw) return QUEST_ERR_NULL;
+    if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+    int s = validate_gemm_shape(M, N, K, bits, bits);
+    if (s) return s;
+    if (!aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < quest_workspace_bytes(M, N, K, bits, bits))
+        return QUEST_ERR_WORKSPACE;
+    if ((s = check_device())) return s;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    Workspace ws = carve_workspace(workspace, M, N, K);
     StageScope scope(QUEST_STAGE_GEMM, st);
     return launch_gemm(ws.a8, ws.b8, ws.rs_a, ws.rs_b, bits, bits, sx, sw, M, N, K, y, y_dtype, N, nullptr, st);
+}
+
+int quest_linear_fwd(const void *x, const void *w, int dtype, int64_t M, int64_t N, int64_t K,
+                     int bits, int had_block, float trust_factor,
+                     void *y, int y_dtype,
+                     uint8_t *xq, float *sx, uint8_t *mx,
+                     uint8_t *wq, float *sw, uint8_t *mw, int w_is_cached,
+                     void *workspace, size_t workspace_bytes, void *stream) {
+    // every argument check of both halves comes before the first launch
+    if (!y) return QUEST_ERR_NULL;
+    if (y_dtype != QUEST_F32 && y_dtype != QUEST_BF16) return QUEST_ERR_DTYPE;
+    if (!aligned(y, y_dtype == QUEST_F32 ? 4 : 2)) return QUEST_ERR_ALIGN;
+    int s = quest_linear_fwd_quantize(x, w, dtype, M, N, K, bits, had_block, trust_factor, xq, sx, mx, wq, sw, mw,
+                                      w_is_cached, workspace, workspace_bytes, stream);
+    if (s) return s;
+    return quest_linear_fwd_contract(sx, sw, M, N, K, bits, y, y_dtype, workspace, workspace_bytes, stream);
 }
 
 // ---- MLP block: three Algorithm-1 layers with the SwiGLU fused into the first contraction -------

@@ -839,6 +839,7 @@ quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
 // otherwise.
 // ---------------------------------------------------------------------------------------------
 constexpr int BLK_TILE_BYTES = 8192;             // per warp: 32 blocks x 256 bytes of bfloat16
+constexpr long long BLOCK_KERNEL_MIN_ELEMS = 32ll << 20;
 
 // Levels, mask bits and packed code words of 32 consecutive rotated elements (16 float2 pairs), for
 // trust_factor >= 1: an element inside the grid is within half a step of its level, so only clipped
@@ -1217,9 +1218,24 @@ int launch_quantize(const QuantJob *jobs, int njobs, int dtype, int64_t cols, in
             if (grid_kind == GRID_FP4 && q.op8) ok = false;
             if (reinterpret_cast<uintptr_t>(q.mask) % 16 != 0 || (q.op8 && reinterpret_cast<uintptr_t>(q.op8) % 16 != 0)) ok = false;
         }
+        {
+            // Below about 32 M elements (a few waves of this kernel's 4096-element warp tasks) the kernels with 32
+            // elements per thread finish a layer sooner: their many short CTAs drain evenly, so the tensor-core
+            // kernel that follows becomes resident earlier (measured on 4096 x 2048 + 2048 x 2048: 31.7 against
+            // 32.9 us per layer; on 16384 x 4096 + 4096 x 4096 this kernel wins, 240.7 against 245.6 us).
+            long long total_elems = 0;
+            for (int j = 0; j < njobs; ++j) total_elems += (long long)jobs[j].rows * cols;
+            if (total_elems < BLOCK_KERNEL_MIN_ELEMS) ok = false;
+        }
         if (ok) {
             const int T = (int)(cols / 128);
-            const int R = T >= 128 ? 1 : 128 / T;                       // rows per CTA: up to 128 threads
+            // rows per CTA.  Rows with a power-of-two number of blocks live inside one warp, so the CTA can be small:
+            // 64 threads with 16 KB of shared memory fit beside a CTA of the tensor-core kernel that is still
+            // draining, which lets the quantizer of the next layer become resident before its predecessor ends.
+            // Other row lengths take as many whole rows as fit in 128 threads.
+            const bool pow2 = (T & (T - 1)) == 0 && T <= 32;
+            const int cta = pow2 ? 64 : 128;
+            const int R = T >= cta ? 1 : cta / T;
             const int threads = (R * T + 31) / 32 * 32;
             const size_t smem = (size_t)(threads / 32) * BLK_TILE_BYTES + sizeof(float) * (size_t)(threads + R);
             for (int j0 = 0; j0 < njobs; j0 += MAX_QUANT_TENSORS) {

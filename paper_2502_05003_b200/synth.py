@@ -11,9 +11,17 @@ import numpy as np
 
 def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
     """Round binary32 to bfloat16 (nearest even); returns the uint16 bit patterns."""
-    w = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
-    rounded = (w + 0x7FFF + ((w >> 16) & 1)) >> 16
-    return rounded.astype(np.uint16)
+    w = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    # w + 0x7FFF + (bit 16 of w), in 32-bit arithmetic: the sum fits for every finite value and infinity
+    # (at most 0xFF800000 + 0x8000); only NaN patterns at the very top of the range need the wide path
+    if w.size and int(w.max()) >= 0xFFFF0000:
+        w64 = w.astype(np.uint64)
+        return ((w64 + 0x7FFF + ((w64 >> 16) & 1)) >> 16).astype(np.uint16)
+    inc = (w >> np.uint32(16)) & np.uint32(1)
+    inc += np.uint32(0x7FFF)
+    inc += w
+    inc >>= np.uint32(16)
+    return inc.astype(np.uint16)
 
 
 def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:

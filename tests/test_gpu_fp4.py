@@ -47,6 +47,12 @@ def test_quantize_bf16_rows_wider_than_8192(g, cols, trust):
     check_quantize(rows("student", 37, cols, g + cols + 1), g, trust)
 
 
+@pytest.mark.parametrize("cols", [2048, 5504])
+def test_quantize_large_tensors_one_thread_per_rotation_block(cols):
+    """The kernel that serves dense bfloat16 tensors of 32 Mi elements and more, with the FP4 grid."""
+    check_quantize(rows("gauss", (32 << 20) // cols + 37, cols, cols), 128, 1.0)
+
+
 @pytest.mark.parametrize("trust", [0.0, 0.5, 1.0, 1.3, 3.0])
 def test_trust_factors(trust):
     check_quantize(rows("gauss", 64, 1024, 5), 128, trust)

@@ -90,6 +90,39 @@ def test_config5_points(bits, d, tokens):
         check_linear(p["x"], p["w"], bits, g, 1.0, torch.bfloat16, BF16_OUT_RTOL, sample_rows=rows)
 
 
+def test_large_layer_quantized_by_the_block_kernel():
+    """x and w of 32 Mi elements together: the quantizer launch with one thread per rotation block writes codes,
+    masks and the tensor-core operands of both tensors (8-bit codes stay on the kernels that also sum the rows)."""
+    p = synth.config5_point(7, 16384, 2048)
+    rows = np.random.default_rng(5).choice(16384, 24, replace=False)
+    check_linear(p["x"], p["w"], 4, 128, 1.0, torch.bfloat16, BF16_OUT_RTOL, sample_rows=rows)
+    check_linear(p["x"], p["w"], 2, 128, 1.0, torch.bfloat16, BF16_OUT_RTOL, sample_rows=rows)
+    check_linear(p["x"], p["w"], 8, 128, 1.0, torch.bfloat16, BF16_OUT_RTOL, sample_rows=rows)
+
+
+def test_linear_fwd_in_two_calls_equals_the_single_call():
+    """quest_linear_fwd_quantize followed by quest_linear_fwd_contract is quest_linear_fwd, bit for bit."""
+    import paper_2502_05003_b200 as quest
+    for bits, M, N, K in ((4, 300, 200, 512), (8, 136, 264, 256), (2, 257, 130, 384)):
+        p = synth.config5_point(bits, M, K)
+        x, w = to_dev(p["x"]), to_dev(synth.f32_to_bf16_bits(synth.weights(N, K, np.random.default_rng(bits))))
+        ref = quest.quest_linear_fwd(x, w, bits, 128, 1.0, out_dtype=torch.bfloat16)
+        saved = {k: torch.zeros_like(ref[k]) for k in ("xq", "sx", "mx", "wq", "sw", "mw")}
+        ws = quest.alloc_workspace(M, N, K, bits, bits)
+        y = torch.zeros_like(ref["y"])
+        quest.quest_linear_fwd_quantize(x, w, bits, 128, 1.0, saved, ws)
+        quest.quest_linear_fwd_contract(saved, M, N, K, bits, y, ws)
+        torch.cuda.synchronize()
+        for k in saved:
+            assert torch.equal(saved[k], ref[k]), k
+        assert torch.equal(y, ref["y"])
+        # the second half alone can be repeated: the operands stay in the workspace
+        y.zero_()
+        quest.quest_linear_fwd_contract(saved, M, N, K, bits, y, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(y, ref["y"])
+
+
 def test_linear_fwd_replays_from_a_cuda_graph():
     """Section 5 runs the whole pipeline under a CUDA graph: the call must be capturable (no
     allocation, no synchronisation) and every replay must reproduce the directly launched result."""

@@ -85,6 +85,18 @@ def test_bf16_rows_wider_than_8192(g, cols, bits, trust):
     check(rows_of("student", 37, cols, bits * 31 + g + cols, True), bits, g, trust)
 
 
+@pytest.mark.parametrize("cols,bits,trust", [(2048, 4, 1.0), (2048, 1, 1.3), (2048, 2, 1.0), (2048, 8, 1.0), (128, 4, 1.0),
+                                             (256, 3, 1.0), (1024, 4, 2.0), (4096, 4, 1.0), (640, 4, 1.0), (5504, 4, 1.0),
+                                             (5504, 8, 1.0), (8320, 2, 1.0), (16384, 4, 1.0), (12288, 1, 1.0)])
+def test_large_tensors_one_thread_per_rotation_block(cols, bits, trust):
+    """From 32 Mi elements on, dense bfloat16 tensors with had_block = 128 and trust_factor >= 1 take the kernel in
+    which one thread owns a whole rotation block: rows whose blocks fill part of a warp (cols = 128 .. 4096, block
+    sums combined by shuffles) and rows that span warps or have a number of blocks that is not a power of two
+    (through shared memory), with a ragged last CTA in every case."""
+    rows = (32 << 20) // cols + 37
+    check(rows_of("gauss", rows, cols, cols + bits, True), bits, 128, trust, repeat=1)
+
+
 @pytest.mark.parametrize("trust", [0.0, 0.5, 1.0, 1.25, 1.3, 3.0])
 @pytest.mark.parametrize("bits", [1, 2, 4])
 def test_trust_factors(bits, trust):
