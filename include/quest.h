@@ -335,6 +335,18 @@ int quest_device_status(void *stream);
 int quest_last_device_status(void *stream);
 
 /*
+ * quest_selftest_bounded_wait -- diagnostic (no counterpart in the paper): runs the time-out path of the
+ * kernels' bounded waits on purpose and harmlessly.  A one-warp kernel waits on a barrier that nothing will
+ * complete, with a limit of `limit_cycles` SM clock cycles (1e3 .. 4e9; 2e6 is about a millisecond); the wait
+ * gives up, records the time-out in the device status word and returns; a second wait in the same CTA is
+ * then refused at once.  No fault, no trap, the context stays usable.  After the stream has run it,
+ * quest_device_status returns QUEST_ERR_DEVICE_TIMEOUT once and QUEST_OK from then on.
+ *   report   optional device array of 4 ints: [0] first wait satisfied (expect 0), [1] second wait satisfied
+ *            (expect 0), [2] abort flag of the CTA (expect 1), [3] second wait shorter than the first (expect 1)
+ */
+int quest_selftest_bounded_wait(int64_t limit_cycles, int *report, void *stream);
+
+/*
  * Measurement aid (no counterpart in the paper): per-stage device times.  While enabled, every
  * entry point brackets each of its stages with a pair of CUDA events on the caller's stream.
  * quest_stage_times waits for the events of the most recent call, adds their elapsed times to

@@ -56,6 +56,18 @@ def quest_device_status() -> int:
     return int(_lib.load().quest_device_status(_stream()))
 
 
+def quest_last_device_status() -> int:
+    return int(_lib.load().quest_last_device_status(_stream()))
+
+
+def quest_selftest_bounded_wait(limit_cycles: int = 2_000_000) -> torch.Tensor:
+    """Makes a bounded wait of the kernels run out on purpose (harmless: one warp, a barrier nothing completes).
+    Returns the 4-int device report; afterwards ``quest_device_status()`` is 12 once, then 0."""
+    report = torch.full((4,), -1, dtype=torch.int32, device="cuda")
+    _lib.check(_lib.load().quest_selftest_bounded_wait(limit_cycles, _p(report), _stream()))
+    return report
+
+
 STAGES = ("quant_x", "quant_w", "unpack", "gemm")
 
 

@@ -15,6 +15,7 @@ EXPORTS = (
     "quest_alpha_star_fp4", "quest_quantize_fp4", "quest_lowbit_gemm_fp4", "quest_linear_fwd_fp4",
     "quest_linear_fwd_weight_only", "quest_weight_only_workspace_bytes",
     "quest_mlp_fwd", "quest_mlp_workspace_bytes", "quest_linear_fwd_quantize", "quest_linear_fwd_contract",
+    "quest_selftest_bounded_wait",
 )
 
 _lib = None
@@ -69,6 +70,8 @@ def load() -> ctypes.CDLL:
     L.quest_linear_fwd_quantize.argtypes = [vp, vp, ci, i64, i64, i64, ci, ci, cf, vp, vp, vp, vp, vp, vp, ci, vp, sz, vp]
     L.quest_linear_fwd_contract.restype = ci
     L.quest_linear_fwd_contract.argtypes = [vp, vp, i64, i64, i64, ci, vp, ci, vp, sz, vp]
+    L.quest_selftest_bounded_wait.restype = ci
+    L.quest_selftest_bounded_wait.argtypes = [i64, vp, vp]
     L.quest_mlp_fwd.restype = ci
     L.quest_mlp_fwd.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, ci, ci, cf, vp, vp, ci, vp, vp, sz, vp]
     L.quest_mlp_workspace_bytes.restype = sz

@@ -185,6 +185,13 @@ int quest_device_status(void *stream) {
 
 int quest_last_device_status(void *stream) { return quest_device_status(stream); }
 
+int quest_selftest_bounded_wait(int64_t limit_cycles, int *report, void *stream) {
+    if (limit_cycles < 1000 || limit_cycles > 4000000000ll) return QUEST_ERR_SHAPE;
+    int s = check_device();
+    if (s) return s;
+    return launch_bounded_wait_probe(limit_cycles, report, reinterpret_cast<cudaStream_t>(stream));
+}
+
 int quest_stage_timing(int enable) {
     if (enable && !g_timer.created) {
         for (int i = 0; i < QUEST_NUM_STAGES; ++i)

@@ -100,14 +100,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false if the CTA is aborting or the limit expired (then it records
 // `code` in the device status word and raises the CTA-wide abort flag).
 __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                       int *status, int code) {
+                                       int *status, int code, long long limit_cycles = WAIT_LIMIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 0; it < 0x7fffffffu; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 15u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+            if (clock64() - t0 > limit_cycles) break;
         }
     }
     *abort_flag = 1;
@@ -366,6 +366,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t rank = TWO ? cluster_ctarank() : 0u;
     const bool leader = rank == 0;
     pdl_launch_dependents();
+    if (threadIdx.x == 32) {
+        // the TMA unit fetches a descriptor on first use: start those fetches now, while the kernel sets up
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+        if constexpr (YT) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
+    }
     const int unit = TWO ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;          // tile-loop index
     const int num_units = TWO ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
@@ -890,8 +896,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 
     if constexpr (YT) {
-        // output tiles still on their way out of shared memory
-        if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        // output tiles still on their way out of shared memory: the CTA may retire once the copy engine has read
+        // them (the writes themselves are ordered before the end of the grid)
+        if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
@@ -1004,6 +1011,34 @@ __global__ void rowsum_i8_kernel(const int8_t *__restrict__ a, long long rows, i
     if (lane == 0) out[row] = s;
 }
 
+// Self-test of the bounded wait: one warp waits, with a short limit, on a barrier that nothing will ever
+// complete.  The wait must give up, record its code in the status word, raise the abort flag, and a second
+// wait must then return at once because the CTA is aborting: the path every kernel of the library takes
+// when a copy or a partner CTA fails to arrive, exercised here without any fault.
+__global__ void bounded_wait_probe_kernel(long long limit_cycles, int *status, int *report) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const long long t0 = clock64();
+        const bool first = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, ST_PRODUCER, limit_cycles);
+        const long long t1 = clock64();
+        const bool second = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, ST_MMA, limit_cycles);
+        const long long t2 = clock64();
+        if (report) {
+            report[0] = first ? 1 : 0;                       // 0: the wait gave up
+            report[1] = second ? 1 : 0;                      // 0: refused at once, the CTA is aborting
+            report[2] = abort_flag;
+            report[3] = (t2 - t1) < (t1 - t0) ? 1 : 0;       // the second wait did not run its limit out again
+        }
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1078,6 +1113,14 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
 }
 
 }  // namespace
+
+int launch_bounded_wait_probe(long long limit_cycles, int *report, cudaStream_t st) {
+    int *status = device_status_word();
+    if (!status) return QUEST_ERR_CUDA;
+    bounded_wait_probe_kernel<<<1, 32, 0, st>>>(limit_cycles, status, report);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
+}
 
 // The operand of w and its row sums come first, so that their place does not depend on M: a caller
 // that keeps the workspace can reuse w's operand across calls with different numbers of rows of x.

@@ -149,6 +149,8 @@ int launch_gemm_swiglu(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, 
                        const float *sx, const float *sw_gate, const float *sw_up, int64_t M, int64_t I, int64_t K,
                        void *h, cudaStream_t st);
 
+int launch_bounded_wait_probe(long long limit_cycles, int *report, cudaStream_t st);
+
 // Per-stage event timing (quest_stage_timing): bracket a stage of another translation unit.
 void *stage_begin(int id, cudaStream_t st);
 void stage_end(void *scope);

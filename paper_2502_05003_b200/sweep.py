@@ -11,6 +11,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import os
 
 import torch
 
@@ -95,12 +96,25 @@ def run_point(index: int, bits: int, d: int, tokens: int, g: int, hbm_gbs: float
             "gemm_path": path, "gemm_frac_peak": round(tops / peak, 3)}
 
 
+def measured_peaks():
+    """Denominators: MEASURED_PEAKS.json at the repository root (HBM copy rate; int8 tensor rate taken as twice the
+    measured bf16 burst rate, the nominal ratio), else the stated fallback figures."""
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), 2.0 * float(p["bf16_tflops"]), "measured"
+    return 6650.0, 2.0 * 1590.0, "fallback"
+
+
 def main():
+    hbm, int8, source = measured_peaks()
     ap = argparse.ArgumentParser()
     ap.add_argument("--quick", action="store_true", help="b = 4 only")
-    ap.add_argument("--hbm-gbs", type=float, default=6540.2, help="measured HBM copy rate (denominator)")
-    ap.add_argument("--int8-tops", type=float, default=3358.6, help="2 x measured bf16 burst rate (denominator)")
+    ap.add_argument("--hbm-gbs", type=float, default=hbm, help="HBM copy rate (denominator; default: %s)" % source)
+    ap.add_argument("--int8-tops", type=float, default=int8, help="2 x bf16 burst rate (denominator; default: %s)" % source)
     args = ap.parse_args()
+    print(json.dumps({"denominators": {"hbm_gbs": args.hbm_gbs, "int8_tops": args.int8_tops, "source": source}}), flush=True)
     rows = []
     index = 0
     for bits in ((4,) if args.quick else (1, 2, 3, 4, 8)):
