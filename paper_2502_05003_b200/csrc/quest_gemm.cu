@@ -555,9 +555,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int quarter = warp & 3;
         const int hgrp = (warp - 2) >> 2;              // which half of the tile's (output) columns
         const int cbase = hgrp * CW;
-        // accumulator column of this warp's chunk c0 (0, 32, 64, 96): plain modes take CW consecutive columns;
-        // SwiGLU takes gate columns [64 hgrp, +64) and the up columns of the same outputs, 128 further on
-        auto acc_col = [&](int c0) { return SWIGLU ? (c0 < 64 ? 64 * hgrp + c0 : 128 + 64 * hgrp + (c0 - 64)) : cbase + c0; };
+        // plain modes: a warp takes CW consecutive accumulator columns; SwiGLU: gate columns [64 hgrp, +64) and
+        // the up columns of the same outputs, 128 further on
         const int ep_tid = threadIdx.x - 64;           // 0..255 over the epilogue warps
         int t = 0;
         bool ok = true;
@@ -620,20 +619,23 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // all of this warp's accumulator columns in one go, then hand the TMEM buffer back to
             // the MMA warp before any arithmetic
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
-            uint32_t r[CW];
+            uint32_t r[SWIGLU ? 1 : CW];
+            auto release_tmem = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (TWO) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[buf]), 0));   // the leader's barrier
+                    else mbar_arrive(smem_u32(&tempty_bar[buf]));
+                }
+            };
+            if constexpr (!SWIGLU) {
 #pragma unroll
-            for (int c0 = 0; c0 < CW; c0 += 32) {
-                const int first_out = SWIGLU ? n0 + 64 * hgrp + (c0 & 63) : n0 + cbase + c0;
-                if (first_out < p.N) tmem_ld32_issue(t_row + (uint32_t)acc_col(c0), &r[c0]);     // uniform predicate
-            }
-            tmem_wait_ld();
+                for (int c0 = 0; c0 < CW; c0 += 32)
+                    if (n0 + cbase + c0 < p.N) tmem_ld32_issue(t_row + (uint32_t)(cbase + c0), &r[c0]);     // uniform predicate
+                tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < CW; ++j) pin(r[j]);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if constexpr (TWO) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[buf]), 0));   // the leader's barrier
-                else mbar_arrive(smem_u32(&tempty_bar[buf]));
+                for (int j = 0; j < CW; ++j) pin(r[j]);
+                release_tmem();
             }
             if constexpr (IHT128) {
                 // trust mask and inverse transform of Algorithm 2 on this thread's block of 128: mask, then the inverse
@@ -668,63 +670,67 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
             if constexpr (SWIGLU) {
+                // 64 output columns per thread, in two rounds of 32: gate and up accumulators of the round come out of
+                // tensor memory together (64 registers), the buffer goes back to the MMA warp after the second load
                 const int out0 = n0 + 64 * hgrp;               // first of this thread's 64 output columns
-                if (out0 < p.N) {                              // uniform across the warp
-                    const float2 sx2 = make_float2(sxr, sxr);
-#pragma unroll
-                    for (int c0 = 0; c0 < CW; c0 += 32) {
-                        uint32_t *rc = &r[c0];
-                        const int ac = acc_col(c0);
-                        if (n0 + 64 * hgrp + (c0 & 63) < p.N) {
-                            if (CORR) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    rc[j] = (uint32_t)((int32_t)((uint32_t)p.mul * rc[j] + (uint32_t)rsa + (uint32_t)cbt[ac + j]) >> p.sh);
-                            }
-                            const float2 *sw2 = reinterpret_cast<const float2 *>(swt + ac);
-#pragma unroll
-                            for (int j = 0; j < 32; j += 2) {
-                                const float2 a2 = MX ? make_float2(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]))
-                                                     : make_float2((float)(int32_t)rc[j], (float)(int32_t)rc[j + 1]);
-                                const float2 y2 = __fmul2_rn(__fmul2_rn(sx2, sw2[j >> 1]), a2);
-                                rc[j] = __float_as_uint(y2.x);
-                                rc[j + 1] = __float_as_uint(y2.y);
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) rc[j] = 0u;
-                        }
-                    }
-                    // h = silu(gate) * up, silu(z) = z / (1 + exp(-z)); one rounding to bfloat16.  The exponential and
-                    // the reciprocal are the hardware approximations (a few units of 2^-23 each, no branches):
-                    // exp(-z) overflows to +inf for z < -88, where the quotient is -0 as it should be.
-#pragma unroll
-                    for (int j = 0; j < 64; ++j) {
-                        const float g = __uint_as_float(r[j]), u = __uint_as_float(r[64 + j]);
-                        float e, rc;
-                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(g * -1.4426950408889634f));
-                        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(1.0f + e));
-                        r[j] = __float_as_uint((g * rc) * u);
-                    }
-                    uint8_t *slab = slab_base;
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                const bool live = out0 < p.N;                  // uniform across the warp
+                uint8_t *slab = slab_base;
+                if (live) {
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the slab's last store has read it
                     __syncwarp();
-                    uint8_t *rowp = slab + lane * 128;
-                    const int sw7 = lane & 7;
+                }
+                const float2 sx2 = make_float2(sxr, sxr);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        uint4 q;
-                        __nv_bfloat162 hh;
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j]), __uint_as_float(r[8 * j + 1]));
-                        q.x = *reinterpret_cast<uint32_t *>(&hh);
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2]), __uint_as_float(r[8 * j + 3]));
-                        q.y = *reinterpret_cast<uint32_t *>(&hh);
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 4]), __uint_as_float(r[8 * j + 5]));
-                        q.z = *reinterpret_cast<uint32_t *>(&hh);
-                        hh = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 6]), __uint_as_float(r[8 * j + 7]));
-                        q.w = *reinterpret_cast<uint32_t *>(&hh);
-                        *reinterpret_cast<uint4 *>(rowp + ((j ^ sw7) << 4)) = q;
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t g[32], u[32];
+                    const int gc = 64 * hgrp + 32 * half, uc = 128 + gc;         // accumulator columns: gate, up
+                    const bool part = out0 + 32 * half < p.N;
+                    if (part) {
+                        tmem_ld32_issue(t_row + (uint32_t)gc, g);
+                        tmem_ld32_issue(t_row + (uint32_t)uc, u);
                     }
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) { pin(g[j]); pin(u[j]); }
+                    if (half == 1) release_tmem();
+                    if (part) {
+                        if (CORR) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                g[j] = (uint32_t)((int32_t)((uint32_t)p.mul * g[j] + (uint32_t)rsa + (uint32_t)cbt[gc + j]) >> p.sh);
+                                u[j] = (uint32_t)((int32_t)((uint32_t)p.mul * u[j] + (uint32_t)rsa + (uint32_t)cbt[uc + j]) >> p.sh);
+                            }
+                        }
+                        const float2 *swg = reinterpret_cast<const float2 *>(swt + gc), *swu = reinterpret_cast<const float2 *>(swt + uc);
+                        uint32_t packed[16];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const float2 ag = MX ? make_float2(__uint_as_float(g[j]), __uint_as_float(g[j + 1]))
+                                                 : make_float2((float)(int32_t)g[j], (float)(int32_t)g[j + 1]);
+                            const float2 au = MX ? make_float2(__uint_as_float(u[j]), __uint_as_float(u[j + 1]))
+                                                 : make_float2((float)(int32_t)u[j], (float)(int32_t)u[j + 1]);
+                            const float2 gv = __fmul2_rn(__fmul2_rn(sx2, swg[j >> 1]), ag);
+                            const float2 uv = __fmul2_rn(__fmul2_rn(sx2, swu[j >> 1]), au);
+                            // h = silu(gate) * up, silu(z) = z / (1 + exp(-z)).  The exponential and the reciprocal are the
+                            // hardware approximations (a few units of 2^-23 each, no branches): exp(-z) overflows to +inf
+                            // for z < -88, where the quotient is -0 as it should be.
+                            float e0, e1, r0, r1;
+                            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(gv.x * -1.4426950408889634f));
+                            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(gv.y * -1.4426950408889634f));
+                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(1.0f + e0));
+                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(1.0f + e1));
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn((gv.x * r0) * uv.x, (gv.y * r1) * uv.y);
+                            packed[j >> 1] = *reinterpret_cast<const uint32_t *>(&hh);
+                        }
+                        uint8_t *rowp = slab + lane * 128;
+                        const int sw7 = lane & 7;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            *reinterpret_cast<uint4 *>(rowp + (((half * 4 + j) ^ sw7) << 4)) =
+                                make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                    }
+                }
+                if (live) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) {
