@@ -1062,8 +1062,41 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+// Encoding a tensor map is a driver call of a microsecond or two, and a layer that is called again and again
+// passes the same pointers and shapes every time.  Each host thread keeps the last few descriptors it built, keyed
+// by everything that goes into them (a descriptor is a pure function of its key, so a hit is always valid).
+struct MapKey {
+    const void *base;
+    int64_t d0, d1, pitch;
+    int box0, box1, swizzle, promo;
+    bool operator==(const MapKey &o) const {
+        return base == o.base && d0 == o.d0 && d1 == o.d1 && pitch == o.pitch && box0 == o.box0 && box1 == o.box1 &&
+               swizzle == o.swizzle && promo == o.promo;
+    }
+};
+struct MapCache {
+    static constexpr int N = 16;
+    MapKey key[N];
+    CUtensorMap map[N];
+    int used = 0, next = 0;
+    const CUtensorMap *find(const MapKey &k) const {
+        for (int i = 0; i < used; ++i)
+            if (key[i] == k) return &map[i];
+        return nullptr;
+    }
+    void put(const MapKey &k, const CUtensorMap &m) {
+        key[next] = k;
+        map[next] = m;
+        next = (next + 1) % N;
+        if (used < N) ++used;
+    }
+};
+static thread_local MapCache t_map_cache;
+
 // int8 matrix [rows x K], K contiguous; box = 128 bytes of K x box_rows rows, 128-byte swizzle.
 int make_operand_map(CUtensorMap *tm, const int8_t *base, int64_t rows, int64_t K, int box_rows) {
+    const MapKey mk = {base, K, rows, K, BK, box_rows, 1, 1};
+    if (const CUtensorMap *hit = t_map_cache.find(mk)) { *tm = *hit; return QUEST_OK; }
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return cuda_fail_msg("cuTensorMapEncodeTiled entry point not available");
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
@@ -1074,11 +1107,14 @@ int make_operand_map(CUtensorMap *tm, const int8_t *base, int64_t rows, int64_t 
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail_msg("cuTensorMapEncodeTiled failed");
+    t_map_cache.put(mk, *tm);
     return QUEST_OK;
 }
 
 // y viewed as bytes: [rows x row_bytes], row pitch pitch_bytes; box = 128 bytes x 32 rows, 128-byte swizzle.
 int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes, int64_t pitch_bytes) {
+    const MapKey mk = {base, row_bytes, rows, pitch_bytes, 128, 32, 1, 0};
+    if (const CUtensorMap *hit = t_map_cache.find(mk)) { *tm = *hit; return QUEST_OK; }
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return cuda_fail_msg("cuTensorMapEncodeTiled entry point not available");
     cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
@@ -1088,6 +1124,7 @@ int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes
     CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cuda_fail_msg("cuTensorMapEncodeTiled failed for the output");
+    t_map_cache.put(mk, *tm);
     return QUEST_OK;
 }
 
