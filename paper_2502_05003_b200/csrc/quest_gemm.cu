@@ -25,7 +25,7 @@
 //
 // Kernel structure:
 //   warp 0      TMA producer: 128B-swizzled K-major tiles of A (128 x 128 B) and B (BN or BN/2 rows
-//               x 128 B) into a 3..5-stage shared-memory ring, completion on mbarriers
+//               x 128 B) into a 3..6-stage shared-memory ring, completion on mbarriers
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128 or 256, N=BN, K=32) x 4 per stage
 //               into one of two TMEM accumulator buffers; tcgen05.commit releases the stage /
 //               signals the epilogue
@@ -290,21 +290,30 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t *r) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void pin(uint32_t &v) { asm volatile("" : "+r"(v)::"memory"); }
 
-template <int BN, bool TWO>
+// Shared memory of a CTA, from a 1024-byte-aligned base: output staging, barriers, the column-scale tiles (and the
+// column corrections of 8-bit codes, CBT), then the operand ring.  The ring takes as many stages as the launch's
+// dynamic shared memory holds behind the alignment padding, up to MAX_NSTAGES: the kernel counts them at run time
+// (a pair kernel with 256 columns gets six when the base needs no padding and no correction tile is wanted, else
+// five).  A lone pair saturates with four stages; with every pair loading, the fifth is worth 4-9 % and the sixth
+// another 1-2 %.
+constexpr int SMEM_OPTIN_MAX = 232448;           // largest dynamic shared memory of a CTA on this part
+template <int BN, bool TWO, bool CBT>
 struct SmemLayout {
-    static constexpr int NSTAGES = TWO ? 5 : (BN == 256 ? 3 : STAGES);   // a lone pair saturates with four; with every pair loading, the fifth is worth 9 % on large shapes
+    static constexpr int MAX_NSTAGES = TWO ? MAX_STAGES : (BN == 256 ? 3 : STAGES);
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_ROWS = TWO ? BN / 2 : BN;         // rows of B this CTA stages
     static constexpr int B_BYTES = B_ROWS * BK;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int BAR_OFFSET = NSTAGES * STAGE_BYTES;
-    static constexpr int STG_OFFSET = BAR_OFFSET;            // [8 warps][SLABS][32 rows x 128 B] output staging
-    static constexpr int SLABS = (BN == 128) ? 2 : 1;           // what the stages leave room for
+    static constexpr int SLABS = (BN == 128) ? 2 : 1;        // what the stages leave room for
+    static constexpr int STG_OFFSET = 0;                     // [8 warps][SLABS][32 rows x 128 B] output staging
     static constexpr int STG_BYTES = EPI_WARPS * SLABS * 4096;
     static constexpr int BAR_OFFSET2 = STG_OFFSET + STG_BYTES;
     static constexpr int SW_OFFSET = BAR_OFFSET2 + 256;      // [2][BN] column scales
     static constexpr int CB_OFFSET = SW_OFFSET + 2 * BN * 4; // [2][BN] column corrections (8-bit codes)
-    static constexpr int TOTAL = CB_OFFSET + 2 * BN * 4 + 1024;   // + slack for 1024-byte alignment
+    static constexpr int RING_OFFSET = (CB_OFFSET + (CBT ? 2 * BN * 4 : 0) + 1023) / 1024 * 1024;
+    static constexpr int WANTED = RING_OFFSET + MAX_NSTAGES * STAGE_BYTES + 1024;   // + slack for 1024-byte alignment
+    static constexpr int TOTAL = WANTED > SMEM_OPTIN_MAX ? SMEM_OPTIN_MAX : WANTED;
+    static_assert(RING_OFFSET + 2 * STAGE_BYTES + 1024 <= TOTAL, "at least two stages must fit");
 };
 
 // YT: y leaves through shared memory and TMA tile stores (whole 128-byte row segments per
@@ -330,7 +339,7 @@ template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
-    using L = SmemLayout<BN, TWO>;
+    using L = SmemLayout<BN, TWO, MODE == 1>;
     constexpr bool CORR = MODE == 1;
     constexpr bool BWD = MODE == 2 || MODE == 3;
     constexpr bool F16 = MODE >= 2;               // bfloat16 operands, binary32 accumulators
@@ -344,10 +353,24 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
     static_assert(!SWIGLU || (BN == 256 && YT && (MODE == 0 || MODE == 1 || MODE == 5)), "SwiGLU epilogue: integer modes, 256 columns, TMA stores");
     constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
-    constexpr int STAGES = L::NSTAGES;
     constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 1024-byte aligned, still a shared pointer
+    // stages of the operand ring that fit behind the padding (the same in every CTA of the launch: the base is a
+    // property of the kernel image)
+    int STAGES;
+    {
+        uint32_t dyn;
+        asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+        const int room = (int)dyn - (int)(smem - smem_raw) - L::RING_OFFSET;
+        STAGES = room / L::STAGE_BYTES;
+        if (STAGES > L::MAX_NSTAGES) STAGES = L::MAX_NSTAGES;
+        if (STAGES < 2) {                        // a launch with too little shared memory: refuse, touch nothing
+            if (threadIdx.x == 0) atomicExch(p.status, ST_PRODUCER);
+            return;
+        }
+    }
+    uint8_t *ring = smem + L::RING_OFFSET;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET2);
     uint64_t *full_bar = bars;                   // [STAGES] TMA -> MMA
     uint64_t *empty_bar = bars + MAX_STAGES;     // [STAGES] MMA -> TMA
@@ -442,7 +465,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ok = mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abort_flag, p.status, ST_PRODUCER);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(&full_bar[stage]);
-                    uint8_t *sa = smem + stage * L::STAGE_BYTES;
+                    uint8_t *sa = ring + stage * L::STAGE_BYTES;
                     // K-major: one box of 128 bytes of K x rows.  MN-major: 64 x 64 chunks (128 bytes of the
                     // M / N dimension x 64 k), 8192 bytes each, in the order of the M / N dimension.
                     if constexpr (TWO) {
@@ -515,7 +538,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ok = mbar_wait(smem_u32(&full_bar[stage]), phase, abort_flag, p.status, ST_MMA);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + stage * L::STAGE_BYTES);
+                    const uint32_t sa = smem_u32(ring + stage * L::STAGE_BYTES);
                     const uint64_t a_desc = AMN ? make_smem_desc_mn(sa) : make_smem_desc(sa);
                     const uint64_t b_desc = BMN ? make_smem_desc_mn(sa + L::A_BYTES) : make_smem_desc(sa + L::A_BYTES);
 #pragma unroll
@@ -1131,7 +1154,7 @@ int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes
 template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
                    cudaStream_t st) {
-    using L = SmemLayout<BN, TWO>;
+    using L = SmemLayout<BN, TWO, MODE == 1>;
     static DynamicSmemOnce smem_attr;            // per kernel instantiation, per device
     {
         cudaError_t e = smem_attr.set(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU>, L::TOTAL);
