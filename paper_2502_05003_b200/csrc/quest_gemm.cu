@@ -299,7 +299,7 @@ __device__ __forceinline__ void pin(uint32_t &v) { asm volatile("" : "+r"(v)::"m
 constexpr int SMEM_OPTIN_MAX = 232448;           // largest dynamic shared memory of a CTA on this part
 template <int BN, bool TWO, bool CBT>
 struct SmemLayout {
-    static constexpr int MAX_NSTAGES = TWO ? MAX_STAGES : (BN == 256 ? 3 : STAGES);
+    static constexpr int MAX_NSTAGES = TWO ? MAX_STAGES : STAGES;     // a single CTA with 256 columns (48 KB stages) gets four when the base needs no padding, else three
     static constexpr int A_BYTES = BM * BK;
     static constexpr int B_ROWS = TWO ? BN / 2 : BN;         // rows of B this CTA stages
     static constexpr int B_BYTES = B_ROWS * BK;
