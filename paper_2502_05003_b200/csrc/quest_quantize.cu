@@ -664,15 +664,18 @@ __device__ __forceinline__ void butterfly32_in_registers(float2 (&v)[16]) {
     }
 }
 
-template <int CB, bool FAST, int GRID = GRID_UNIFORM>
+// G (threads per rotation block) is a template parameter so that every index of the two layout changes is a
+// compile-time offset.
+template <int CB, bool FAST, int GRID, int G>
 __global__ void __launch_bounds__(256, 3)
 quantize_wide_kernel(const __grid_constant__ QuantArgs a, int exchange_bytes) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     pdl_launch_dependents();
     pdl_wait();
     const int cols = a.cols, S = a.S, R = a.R;
-    const int G = a.had_block >> 5;                            // threads per rotation block: 32, 64 or 128
-    const int gshift = 31 - __clz(G);
+    static_assert(G == 32 || G == 64 || G == 128, "rotation blocks of 1024, 2048 or 4096 elements");
+    constexpr int gshift = G == 32 ? 5 : G == 64 ? 6 : 7;
+    constexpr int GBLOCK = 32 * G;                             // elements of a rotation block
     float *xsm = reinterpret_cast<float *>(smem_raw);
     float *tbuf = reinterpret_cast<float *>(smem_raw + exchange_bytes);
     const int trow_words = cols + (cols >> 3);                 // 36 words per 32 elements
@@ -680,7 +683,7 @@ quantize_wide_kernel(const __grid_constant__ QuantArgs a, int exchange_bytes) {
     const int r_local = tid / S;
     const int tr = tid - r_local * S;
     const int p = tr & (G - 1);
-    const int blk_base = (tr >> gshift) * a.had_block;         // first element of this thread's block
+    const int blk_base = (tr >> gshift) * GBLOCK;              // first element of this thread's block
     {
         const int grp = (int)blockIdx.x;                       // one CTA per group of R rows
         const int which = grp >= a.blocks0 ? 1 : 0;
@@ -702,25 +705,27 @@ quantize_wide_kernel(const __grid_constant__ QuantArgs a, int exchange_bytes) {
             }
             butterfly32_in_registers(v);
             float *trow = tbuf + (size_t)r_local * trow_words;
+            // element i sits at word i + 4 (i / 32); with i = blk_base + p + G j and G a multiple of 32 that is a base
+            // plus j (G + G / 8)
+            float *tdst = trow + (blk_base + p) + (((blk_base + p) >> 5) << 2);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                const int i0 = blk_base + p + ((2 * j) << gshift), i1 = blk_base + p + ((2 * j + 1) << gshift);
-                trow[i0 + ((i0 >> 5) << 2)] = v[j].x;
-                trow[i1 + ((i1 >> 5) << 2)] = v[j].y;
+                tdst[(2 * j) * (G + G / 8)] = v[j].x;
+                tdst[(2 * j + 1) * (G + G / 8)] = v[j].y;
             }
         }
         __syncthreads();
         {   // phase B: 32 contiguous elements; strides g/64 .. 32 against the partner threads' elements
             const float *trow = tbuf + (size_t)r_local * trow_words;
             const float4 *own = reinterpret_cast<const float4 *>(trow + tr * 36);
-            if (G == 32) {
+            if constexpr (G == 32) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 o = own[q];
                     v[2 * q] = make_float2(o.x, o.y);
                     v[2 * q + 1] = make_float2(o.z, o.w);
                 }
-            } else if (G == 64) {
+            } else if constexpr (G == 64) {
                 const float4 *p1 = reinterpret_cast<const float4 *>(trow + (tr ^ 1) * 36);
                 const float s1 = (tr & 1) ? -1.0f : 1.0f;
                 const float2 sg1 = make_float2(s1, s1);
@@ -754,15 +759,15 @@ quantize_wide_kernel(const __grid_constant__ QuantArgs a, int exchange_bytes) {
     }
 }
 
-template <int GRID, bool FAST>
-static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
-                               int exchange_bytes) {
+template <int GRID, bool FAST, int G>
+static cudaError_t launch_wide_g(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                                 int exchange_bytes) {
 #define QUEST_LAUNCH(CBV)                                                                                   \
     do {                                                                                                    \
         static DynamicSmemOnce once_;                                                                       \
-        cudaError_t e_ = once_.set(quantize_wide_kernel<CBV, FAST, GRID>, 160 * 1024);                      \
+        cudaError_t e_ = once_.set(quantize_wide_kernel<CBV, FAST, GRID, G>, 160 * 1024);                   \
         if (e_ != cudaSuccess) return e_;                                                                   \
-        return launch_pdl(quantize_wide_kernel<CBV, FAST, GRID>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
+        return launch_pdl(quantize_wide_kernel<CBV, FAST, GRID, G>, dim3((unsigned)grid), dim3(threads), smem, st, 1, a, \
                           exchange_bytes);                                                                  \
     } while (0)
     if (GRID == GRID_FP4) QUEST_LAUNCH(4);
@@ -773,6 +778,16 @@ static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaS
         default: QUEST_LAUNCH(8);
     }
 #undef QUEST_LAUNCH
+}
+
+template <int GRID, bool FAST>
+static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                               int exchange_bytes) {
+    switch (a.had_block) {
+        case 1024: return launch_wide_g<GRID, FAST, 32>(cb, grid, threads, smem, st, a, exchange_bytes);
+        case 2048: return launch_wide_g<GRID, FAST, 64>(cb, grid, threads, smem, st, a, exchange_bytes);
+        default: return launch_wide_g<GRID, FAST, 128>(cb, grid, threads, smem, st, a, exchange_bytes);
+    }
 }
 
 // The specialised case (bfloat16 rows, had_block = 128, 32 elements per thread) with direct loads and

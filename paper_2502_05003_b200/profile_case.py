@@ -2,6 +2,7 @@
 
     python -m paper_2502_05003_b200.profile_case linear [calls]      # quest_linear_fwd, X[4096 x 2048] W[2048 x 2048], b = 4
     python -m paper_2502_05003_b200.profile_case quantize-large      # quest_quantize alone: 6144 x 5504 and 8192 x 4096
+    python -m paper_2502_05003_b200.profile_case quantize-wide       # quest_quantize alone, 8192 x 4096, one rotation block per row
     python -m paper_2502_05003_b200.profile_case mlp                 # quest_mlp_fwd, 4096 tokens, H = 2048, I = 5504
     python -m paper_2502_05003_b200.profile_case backward [calls]    # quest_linear_bwd on the config-2 layer
 
@@ -42,6 +43,17 @@ def quantize_large() -> None:
             quest.quest_quantize(x, 4, 128, 1.0, codes=c, scales=s, mask=m)
 
 
+def quantize_wide() -> None:
+    dev = torch.device("cuda")
+    rows, cols = 8192, 4096
+    x = torch.randn(rows, cols, device=dev).bfloat16()
+    c = torch.empty(rows, cols // 2, dtype=torch.uint8, device=dev)
+    s = torch.empty(rows, device=dev)
+    m = torch.empty(rows, cols // 8, dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        quest.quest_quantize(x, 4, cols, 1.0, codes=c, scales=s, mask=m)
+
+
 def mlp() -> None:
     T, H, I = 4096, 2048, 5504
     dev = torch.device("cuda")
@@ -74,6 +86,8 @@ def main() -> None:
         linear(n or 6)
     elif case == "quantize-large":
         quantize_large()
+    elif case == "quantize-wide":
+        quantize_wide()
     elif case == "mlp":
         mlp()
     elif case == "backward":
