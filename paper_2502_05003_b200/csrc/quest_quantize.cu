@@ -197,7 +197,8 @@ __device__ __forceinline__ uint32_t cvt_e2m1x8(const float (&t)[8]) {
 // one warp, codes, scales and mask requested (the GEMM operand and the bfloat16 outputs of the
 // weight-only variant are optional; a tensor may also ask for the rotation alone), no row sums,
 // trust_factor >= 1 -- so that no per-row loop and only a few uniform branches remain.
-template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false, bool RS = false>
+// CS, CCOLS: threads per row and row length when the kernel is instantiated for one row length (0 = run-time values).
+template <int CB, int E, bool GFULL, bool FAST, int GRID = GRID_UNIFORM, bool XDONE = false, bool RS = false, int CS = 0, int CCOLS = 0>
 __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const QuantArgs &a, const QuantTensor &tn,
                                                      bool active, long long row, int tr, int r_local, float *xsm,
                                                      int s_start) {
@@ -205,8 +206,8 @@ __device__ __forceinline__ void rotate_project_store(float2 (&v)[E / 2], const Q
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int nthreads = blockDim.x;
-    const int S = a.S;
-    const int cols = a.cols;
+    const int S = CS ? CS : a.S;
+    const int cols = CCOLS ? CCOLS : a.cols;
     const int had_block = a.had_block;
     // ---- rotation, descending stride --------------------------------------------------------
     const float2 neg1 = make_float2(-1.0f, -1.0f);
@@ -795,9 +796,13 @@ static cudaError_t launch_wide(int cb, int grid, int threads, size_t smem, cudaS
 // scheduling balances better than the persistent loop of the streaming kernel and there is no
 // staging to set up.  Stride 64 pairs this thread with lane ^ 2 (shuffles); the rest is the common tail.
 // RS: the row sums of the 8-bit GEMM operand are wanted (kept out of the common instantiation).
-template <int CB, int GRID = GRID_UNIFORM, bool RS = false>
+// COLS: the row length when it is one of the common ones (1024, 2048, 4096: threads per row, rows per CTA and every
+// row pitch become constants, worth 6 % of the kernel); 0 takes them from the arguments.
+template <int CB, int GRID = GRID_UNIFORM, bool RS = false, int COLS = 0>
 __global__ void __launch_bounds__(256, 4)
 quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
+    constexpr int CS = COLS / 32;
+    const int S = CS ? CS : a.S, R = CS ? 128 / CS : a.R, cols = COLS ? COLS : a.cols;
     extern __shared__ float xsm[];                 // [warps] partial sums
     pdl_launch_dependents();
     pdl_wait();
@@ -805,10 +810,10 @@ quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
     const int which = (int)blockIdx.x >= a.blocks0 ? 1 : 0;
     const QuantTensor &tn = a.t[which];
     const int blk = which ? (int)blockIdx.x - a.blocks0 : (int)blockIdx.x;
-    const int r_local = tid / a.S;
-    const int tr = tid - r_local * a.S;
-    const long long row = (long long)blk * a.R + r_local;
-    const bool active = row < tn.rows && tr < (a.cols >> 5);   // slots past the row end hold zeros
+    const int r_local = tid / S;
+    const int tr = tid - r_local * S;
+    const long long row = (long long)blk * R + r_local;
+    const bool active = row < tn.rows && tr < (cols >> 5);     // slots past the row end hold zeros
     float2 v[16];
     if (active) {
         const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(tn.x) + row * tn.ld + (long long)tr * 32);
@@ -835,7 +840,7 @@ quantize_direct128_kernel(const __grid_constant__ QuantArgs a) {
             v[i] = __ffma2_rn(v[i], sgn, p);
         }
     }
-    rotate_project_store<CB, 32, true, true, GRID, false, RS>(v, a, tn, active, row, tr, r_local, xsm, 32);
+    rotate_project_store<CB, 32, true, true, GRID, false, RS, CS, COLS>(v, a, tn, active, row, tr, r_local, xsm, 32);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1138,17 +1143,30 @@ static cudaError_t launch_block128(int cb, dim3 grid, int threads, size_t smem, 
     }
 }
 
+template <int GRID, int COLS>
+static cudaError_t launch_direct128_cols(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
+                                         bool rowsums) {
+    if (rowsums) return launch_pdl(quantize_direct128_kernel<8, GRID_UNIFORM, true, COLS>, grid, dim3(threads), smem, st, 1, a);
+    if (GRID == GRID_FP4) return launch_pdl(quantize_direct128_kernel<4, GRID, false, COLS>, grid, dim3(threads), smem, st, 1, a);
+    switch (cb) {
+        case 1: return launch_pdl(quantize_direct128_kernel<1, GRID, false, COLS>, grid, dim3(threads), smem, st, 1, a);
+        case 2: return launch_pdl(quantize_direct128_kernel<2, GRID, false, COLS>, grid, dim3(threads), smem, st, 1, a);
+        case 4: return launch_pdl(quantize_direct128_kernel<4, GRID, false, COLS>, grid, dim3(threads), smem, st, 1, a);
+        default: return launch_pdl(quantize_direct128_kernel<8, GRID, false, COLS>, grid, dim3(threads), smem, st, 1, a);
+    }
+}
+
 template <int GRID>
 static cudaError_t launch_direct128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a,
                                     bool rowsums = false) {
-    if (rowsums) return launch_pdl(quantize_direct128_kernel<8, GRID_UNIFORM, true>, grid, dim3(threads), smem, st, 1, a);
-    if (GRID == GRID_FP4) return launch_pdl(quantize_direct128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
-    switch (cb) {
-        case 1: return launch_pdl(quantize_direct128_kernel<1, GRID>, grid, dim3(threads), smem, st, 1, a);
-        case 2: return launch_pdl(quantize_direct128_kernel<2, GRID>, grid, dim3(threads), smem, st, 1, a);
-        case 4: return launch_pdl(quantize_direct128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
-        default: return launch_pdl(quantize_direct128_kernel<8, GRID>, grid, dim3(threads), smem, st, 1, a);
+    // the instantiations for one row length assume the launch geometry chosen for it: cols / 32 threads per row,
+    // CTAs of 128 threads
+    if (threads == 128 && a.S * 32 == a.cols && a.R * a.S == 128) {
+        if (a.cols == 1024) return launch_direct128_cols<GRID, 1024>(cb, grid, threads, smem, st, a, rowsums);
+        if (a.cols == 2048) return launch_direct128_cols<GRID, 2048>(cb, grid, threads, smem, st, a, rowsums);
+        if (a.cols == 4096) return launch_direct128_cols<GRID, 4096>(cb, grid, threads, smem, st, a, rowsums);
     }
+    return launch_direct128_cols<GRID, 0>(cb, grid, threads, smem, st, a, rowsums);
 }
 
 template <bool BF16, int E>
