@@ -948,9 +948,13 @@ __device__ __forceinline__ void tile_to_global(const uint8_t *tile, uint8_t *dst
     }
 }
 
-template <int CB, int GRID>
+// CT: blocks per row when the kernel is instantiated for one row length (16, 32 and 43 blocks: 2048, 4096 and 5504
+// columns); 0 takes the row length and the rows per CTA from the arguments.
+template <int CB, int GRID, int CT = 0>
 __global__ void __launch_bounds__(128, 3)
 quantize_block128_kernel(const __grid_constant__ QuantArgs a) {
+    constexpr bool CT_POW2 = CT != 0 && (CT & (CT - 1)) == 0 && CT <= 32;
+    constexpr int CR = CT == 0 ? 0 : CT_POW2 ? 64 / CT : (CT >= 128 ? 1 : 128 / CT);     // the host's choice of rows per CTA
     extern __shared__ __align__(16) uint8_t smem_raw[];   // [warps][8 KB] tiles, then [threads] + [rows] floats
     pdl_launch_dependents();
     pdl_wait();
@@ -959,11 +963,12 @@ quantize_block128_kernel(const __grid_constant__ QuantArgs a) {
     const int which = (bid >= a.bend[0] ? 1 : 0) + (bid >= a.bend[1] ? 1 : 0) + (bid >= a.bend[2] ? 1 : 0);
     const QuantTensor &tn = a.t[which];
     const int blk = which ? bid - a.bend[which - 1] : bid;
-    const int cols = a.cols;
-    const int T = cols >> 7;                                   // blocks (= threads) per row
-    const long long row0 = (long long)blk * a.R;
+    const int cols = CT ? CT * 128 : a.cols;
+    const int T = CT ? CT : cols >> 7;                         // blocks (= threads) per row
+    const int R = CT ? CR : a.R;
+    const long long row0 = (long long)blk * R;
     const long long rows_left = tn.rows - row0;
-    const int rows_here = rows_left < a.R ? (int)rows_left : a.R;
+    const int rows_here = rows_left < R ? (int)rows_left : R;
     const int nslots = rows_here * T;                          // live (row, block) slots of this CTA
     const bool active = tid < nslots;
     uint8_t *tile = smem_raw + warp * BLK_TILE_BYTES;
@@ -1129,18 +1134,27 @@ quantize_block128_kernel(const __grid_constant__ QuantArgs a) {
     }
 }
 
-template <int GRID>
-static cudaError_t launch_block128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
+template <int GRID, int CT>
+static cudaError_t launch_block128_ct(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
     if constexpr (GRID == GRID_FP4) {
-        return launch_pdl(quantize_block128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
+        return launch_pdl(quantize_block128_kernel<4, GRID, CT>, grid, dim3(threads), smem, st, 1, a);
     } else {
         switch (cb) {
-            case 1: return launch_pdl(quantize_block128_kernel<1, GRID>, grid, dim3(threads), smem, st, 1, a);
-            case 2: return launch_pdl(quantize_block128_kernel<2, GRID>, grid, dim3(threads), smem, st, 1, a);
-            case 4: return launch_pdl(quantize_block128_kernel<4, GRID>, grid, dim3(threads), smem, st, 1, a);
-            default: return launch_pdl(quantize_block128_kernel<8, GRID>, grid, dim3(threads), smem, st, 1, a);
+            case 1: return launch_pdl(quantize_block128_kernel<1, GRID, CT>, grid, dim3(threads), smem, st, 1, a);
+            case 2: return launch_pdl(quantize_block128_kernel<2, GRID, CT>, grid, dim3(threads), smem, st, 1, a);
+            case 4: return launch_pdl(quantize_block128_kernel<4, GRID, CT>, grid, dim3(threads), smem, st, 1, a);
+            default: return launch_pdl(quantize_block128_kernel<8, GRID, CT>, grid, dim3(threads), smem, st, 1, a);
         }
     }
+}
+
+template <int GRID>
+static cudaError_t launch_block128(int cb, dim3 grid, int threads, size_t smem, cudaStream_t st, const QuantArgs &a) {
+    // the instantiations for one row length assume the rows per CTA the host derives from it
+    if (a.cols == 2048 && a.R == 4) return launch_block128_ct<GRID, 16>(cb, grid, threads, smem, st, a);
+    if (a.cols == 4096 && a.R == 2) return launch_block128_ct<GRID, 32>(cb, grid, threads, smem, st, a);
+    if (a.cols == 5504 && a.R == 2) return launch_block128_ct<GRID, 43>(cb, grid, threads, smem, st, a);
+    return launch_block128_ct<GRID, 0>(cb, grid, threads, smem, st, a);
 }
 
 template <int GRID, int COLS>
