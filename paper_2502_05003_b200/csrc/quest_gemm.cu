@@ -219,6 +219,14 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves of the cluster barrier on their own: a warp arrives as soon as it has nothing left to publish to
+// the peer CTA and waits only where it needs the peer, so the barrier's latency overlaps the work between.
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
@@ -335,7 +343,11 @@ struct SmemLayout {
 // projection (the B operand stacks the rows of w_gate and w_up), every epilogue thread holds gate and
 // up of 64 output columns of its row, and the tile leaves as h = silu(gate) * up in bfloat16: the
 // MLP block's gate and up products never reach memory.
-template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false>
+// SHORT (pair kernels of mode 0 with bfloat16 output through TMA stores and no raw accumulators): the instantiation
+// for launches in which a CTA pair runs at most two tiles, where set-up and exit are a visible share.  Each warp
+// arrives at the two cluster barriers as early as it can and waits as late as it can, and the output type and the
+// absence of the accumulator output are constants.  With many tiles per pair the plain form measured faster.
+template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false, bool SHORT = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmY, GemmParams p) {
@@ -352,6 +364,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     static_assert(OPL == 0 || MODE == 2 || MODE == 3, "MN-major operands: bfloat16 backward modes only");
     static_assert(!IHT128 || BN == 256, "the fused inverse transform needs 128 columns per thread");
     static_assert(!SWIGLU || (BN == 256 && YT && (MODE == 0 || MODE == 1 || MODE == 5)), "SwiGLU epilogue: integer modes, 256 columns, TMA stores");
+    static_assert(!SHORT || (TWO && MODE == 0 && YT && !SWIGLU && OPL == 0), "the short-launch form: plain int8 pair kernel");
     constexpr int BN_OUT = SWIGLU ? BN / 2 : BN;  // output columns per tile
     constexpr int TILE_M = TWO ? 2 * BM : BM;    // rows of one output tile (both CTAs of a pair)
     extern __shared__ uint8_t smem_raw[];
@@ -411,6 +424,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // barriers visible to the TMA unit
     }
+    if constexpr (SHORT) {
+        // only warp 0 has something to publish to the peer (the initialised barriers): every warp arrives at the
+        // cluster barrier now and waits after the TMEM allocation
+        __syncwarp();
+        cluster_arrive();
+    }
     if (warp == 1) {
         if constexpr (TWO) {      // executed by this warp of both CTAs of the pair
             asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -426,7 +445,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if constexpr (TWO) cluster_sync_all();       // the peer's barriers are initialised before anything signals them
+    if constexpr (SHORT) cluster_wait();         // the peer's barriers are initialised before anything signals them
+    else if constexpr (TWO) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     if constexpr (MX) {
@@ -449,6 +469,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int num_n = (p.N + BN_OUT - 1) / BN_OUT;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
+    // SHORT, leaving: a CTA must stay until its peer can no longer signal its barriers or read its shared and tensor
+    // memory.  An epilogue warp arrives at the cluster barrier right after handing back its last accumulator buffer
+    // (its last signal to the peer), the other warps after their loops, and everyone waits at the very end.
+    [[maybe_unused]] bool left = false;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -585,8 +609,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         const bool vec_y = p.y && (((reinterpret_cast<uintptr_t>(p.y) & 15) == 0) &&
                                    (p.ldy % (p.y_dtype == QUEST_BF16 ? 8 : 4) == 0));
-        const bool vec_acc = p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
-        const bool y_f32 = p.y_dtype == QUEST_F32;
+        const bool vec_acc = !SHORT && p.acc && (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.acc) & 15) == 0);
+        const bool y_f32 = !SHORT && p.y_dtype == QUEST_F32;
         uint8_t *slab_base = smem + L::STG_OFFSET + (warp - 2) * (L::SLABS * 4096);
         int slab_count = 0;                            // slabs this warp has handed to TMA
         for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++t) {
@@ -617,7 +641,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool row_ok = row < p.M;
             // without 8-bit corrections and without the raw accumulators, the exact power of two of the
             // operand scaling is folded into the row scale instead of shifting every accumulator
-            const bool fold = !CORR && !p.acc;
+            const bool fold = SHORT || (!CORR && !p.acc);
             float sxr = WO ? 1.0f : (!BWD && row_ok && p.y) ? __ldg(p.sx + row) : 0.0f;
             if (fold) sxr = __fmul_rn(sxr, __uint_as_float((uint32_t)(127 - p.sh) << 23));
             int rsa = 0;
@@ -649,6 +673,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (lane == 0) {
                     if constexpr (TWO) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[buf]), 0));   // the leader's barrier
                     else mbar_arrive(smem_u32(&tempty_bar[buf]));
+                }
+                if constexpr (SHORT) {
+                    if (tile + num_units >= num_tiles) {       // this CTA's last tile: nothing more goes to the peer
+                        __syncwarp();
+                        cluster_arrive();
+                        left = true;
+                    }
                 }
             };
             if constexpr (!SWIGLU) {
@@ -805,7 +836,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 if (col0 + j < p.N) dst[j] = __float2int_rn(__uint_as_float(rc[j]) * am);
                         }
                     }
-                    if (!MX && !BWD && p.acc && row_ok) {
+                    if (!SHORT && !MX && !BWD && p.acc && row_ok) {
                         int32_t *dst = p.acc + (long long)row * p.N + col0;
                         if (vec_acc && full) {
 #pragma unroll
@@ -930,10 +961,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     }
     tc_fence_before();
-    __syncthreads();
-    // a CTA of a pair must stay until its peer can no longer signal its barriers or read its
-    // shared memory and tensor memory
-    if constexpr (TWO) cluster_sync_all();
+    if constexpr (SHORT) {
+        __syncwarp();
+        if (!left) cluster_arrive();             // uniform per warp
+        cluster_wait();
+    } else {
+        __syncthreads();
+        // a CTA of a pair must stay until its peer can no longer signal its barriers or read its
+        // shared memory and tensor memory
+        if constexpr (TWO) cluster_sync_all();
+    }
     if (warp == 1) {
         tc_fence_after();
         if constexpr (TWO)
@@ -1151,13 +1188,13 @@ int make_output_map(CUtensorMap *tm, void *base, int64_t rows, int64_t row_bytes
     return QUEST_OK;
 }
 
-template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false>
+template <int BN, int MODE, bool TWO, bool YT, int OPL = 0, bool SWIGLU = false, bool SHORT = false>
 int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmY, const GemmParams &p,
                    cudaStream_t st) {
     using L = SmemLayout<BN, TWO, MODE == 1>;
     static DynamicSmemOnce smem_attr;            // per kernel instantiation, per device
     {
-        cudaError_t e = smem_attr.set(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU>, L::TOTAL);
+        cudaError_t e = smem_attr.set(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU, SHORT>, L::TOTAL);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     int dev = 0, sms = 148;
@@ -1173,7 +1210,7 @@ int launch_gemm_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtenso
     } else {
         grid = tiles < sms ? tiles : sms;
     }
-    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
+    cudaError_t e = launch_pdl(gemm_i8_kernel<BN, MODE, TWO, YT, OPL, SWIGLU, SHORT>, dim3((unsigned)grid), dim3(NUM_THREADS), (size_t)L::TOTAL, st,
                                TWO ? 2 : 1, tmA, tmB, tmY, p);
     return e == cudaSuccess ? QUEST_OK : cuda_fail(e);
 }
@@ -1296,6 +1333,14 @@ int launch_gemm(const int8_t *a8, const int8_t *b8, const int32_t *rs_a, const i
                 : launch_gemm_bn<BNV, 1, TWOV, false>(tmA, tmB, tmY, p, st))                           \
           : (yt ? launch_gemm_bn<BNV, 0, TWOV, true>(tmA, tmB, tmY, p, st)                            \
                 : launch_gemm_bn<BNV, 0, TWOV, false>(tmA, tmB, tmY, p, st)))
+    if (pair && !corr && yt && y_dtype == QUEST_BF16 && !acc) {
+        // at most two tiles per CTA pair: the form that hides the cluster barriers of set-up and exit
+        int dev = 0, sms = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int64_t tiles = ((M + 255) / 256) * ((N + 255) / 256);
+        if (tiles <= 2 * (int64_t)(sms / 2)) return launch_gemm_bn<256, 0, true, true, 0, false, true>(tmA, tmB, tmY, p, st);
+    }
     if (pair) return QUEST_GEMM(256, true);
     if (wide) return QUEST_GEMM(256, false);
     return QUEST_GEMM(128, false);
